@@ -15,7 +15,6 @@ from fractions import Fraction
 
 import numpy as np
 import pytest
-import torch
 
 from oracle import cq_oracle as orc
 from paper_2410_07505_b200 import workloads as wl
@@ -44,6 +43,7 @@ def test_decode_f16_all_patterns_matches_numpy():
 
 
 def test_decode_bf16_all_patterns_matches_torch():
+    import torch
     bits = np.arange(65536, dtype=np.uint16)
     got = orc.decode16(bits, "bf16")
     ref = torch.from_numpy(bits.view(np.int16).copy()).view(torch.bfloat16).to(torch.float32).numpy()
@@ -81,6 +81,7 @@ def test_encode_f16_matches_numpy_cast():
 
 
 def test_encode_bf16_matches_torch_cast():
+    import torch
     v = _encode_probe_values()
     ref = torch.from_numpy(v).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
     assert np.array_equal(orc.encode16(v, "bf16"), ref)
