@@ -1,0 +1,148 @@
+/*
+ * cq.h -- C ABI of the CrossQuant activation cross-quantizer for NVIDIA B200 (sm_100a).
+ *
+ * The operations follow the paper "CrossQuant" (arXiv 2410.07505): Eq. 1 (per-token
+ * quantization), Eq. 2 (per-channel weight quantization), Definition 1 (the quantization
+ * kernel: the set of elements whose code is 0) and the CrossQuant equation of Section 4.2,
+ *
+ *     CQ(X_ij) = round( X_ij / D_ij ),   D_ij = t_i^alpha * c_j^(1-alpha) / (2^(N-1) - 1),
+ *     t_i = max_j |X_ij| ,  c_j = max_i |X_ij| ,  0 <= alpha <= 1.
+ *
+ * Conventions that hold for every function unless it says otherwise
+ *   - Matrices are row-major, 16-bit (IEEE binary16 or bfloat16), `ld` = distance between rows
+ *     in elements (ld >= columns).  Sizes are 64-bit.  Inputs are expected to be finite.
+ *   - Every data pointer is a DEVICE pointer owned by the caller.  The library allocates
+ *     nothing, frees nothing and keeps no per-call state.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All work is
+ *     enqueued on it; no call synchronises; scalar results are written to device memory.
+ *   - The return value is a cq_status.  On any status other than CQ_OK no kernel was launched
+ *     by that call (CQ_ERR_CUDA excepted: it reports a launch the driver refused).
+ *   - Arithmetic (identical for every alpha, bit width and shape):
+ *         qmax = 2^(bits-1) - 1
+ *         alpha == 1 : a_i = fl32(t_i / qmax), b_j = 1        (Eq. 1 exactly)
+ *         alpha == 0 : a_i = 1, b_j = fl32(c_j / qmax)        (per-column quantization)
+ *         else       : a_i = fl32(pow_fp64(t_i, alpha) / qmax), b_j = fl32(pow_fp64(c_j, 1-alpha))
+ *         s_ij = fl32(a_i * b_j);  s_ij == 0 -> code 0, dequantized 0
+ *         code = round-half-even(fl32(x_ij / s_ij)) clamped to [-qmax, qmax]
+ *         xhat = fl32(code * s_ij), rounded once more (nearest-even) when a 16-bit output is asked
+ *   - INT4 storage: two codes per byte; element (i, 2k) in the low nibble and (i, 2k+1) in the
+ *     high nibble of byte i*(I/2)+k; two's-complement nibbles in [-7, 7].  I must be even.
+ *   - Fast kernels need 16-byte aligned matrix pointers and I, ld multiples of 8; any other
+ *     shape or alignment (2-byte aligned at least) is served by slower general kernels with
+ *     identical results.
+ */
+#ifndef CQ_H_
+#define CQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    CQ_OK = 0,
+    CQ_ERR_NULL = 1,       /* a required pointer is NULL                                   */
+    CQ_ERR_SHAPE = 2,      /* negative size, ld < columns, or a size beyond what is supported */
+    CQ_ERR_DTYPE = 3,      /* dtype not valid for that argument                            */
+    CQ_ERR_BITS = 4,       /* bits not in {4, 8}                                           */
+    CQ_ERR_ALPHA = 5,      /* alpha outside [0, 1] or NaN                                  */
+    CQ_ERR_ALIGN = 6,      /* pointer not aligned to its element size, or odd I with INT4  */
+    CQ_ERR_WORKSPACE = 7,  /* workspace NULL, misaligned (256 B) or smaller than required  */
+    CQ_ERR_CUDA = 8        /* the CUDA runtime reported an error at launch                 */
+} cq_status;
+
+typedef enum { CQ_F16 = 0, CQ_BF16 = 1, CQ_F32 = 2 /* outputs only */ } cq_dtype;
+
+int cq_version(void);
+const char* cq_status_string(int status);
+
+/* t_i = max_j |X_ij| (Eq. 1).  X: device [T x ld] 16-bit.  t: device float[T], overwritten. */
+int cq_absmax_rows(const void* X, int dtype, int64_t T, int64_t I, int64_t ld, float* t, void* stream);
+
+/* c_j = max_i |X_ij| (CrossQuant equation, Section 4.2).  c: device float[I], overwritten. */
+int cq_absmax_cols(const void* X, int dtype, int64_t T, int64_t I, int64_t ld, float* c, void* stream);
+
+/* Both vectors from a single read of X. */
+int cq_absmax_rows_cols(const void* X, int dtype, int64_t T, int64_t I, int64_t ld,
+                        float* t, float* c, void* stream);
+
+/* Bytes of device workspace cq_quantize_act / cq_kernel_count_x need for a T x I matrix
+ * (scale vectors, their reciprocals and the partial maxima of the first pass). */
+size_t cq_workspace_bytes(int64_t T, int64_t I);
+
+/*
+ * The CrossQuant activation quantizer (Section 4.2): absmax vectors, scale vectors, codes,
+ * dequantized matrix and the size of the quantization kernel (Definition 1), in three launches.
+ *   X          in   device [T x ld], dtype CQ_F16 or CQ_BF16
+ *   alpha      in   exponent of the row maxima, [0, 1]; 1 = per-token (Eq. 1), 0 = per-column
+ *   bits       in   8 or 4
+ *   t, c       out  device float[T], float[I]; nullable
+ *   row_scale  out  device float[T], a_i;  col_scale out device float[I], b_j; nullable
+ *   codes      out  device int8[T*I] (bits = 8) or uint8[T*I/2] (bits = 4); nullable
+ *   deq        out  device [T*I] of deq_dtype (X's dtype or CQ_F32); nullable
+ *   zero_count out  device uint64, number of zero codes = |K(CQ)|; nullable
+ *   workspace  in   device, 256-byte aligned, >= cq_workspace_bytes(T, I); contents undefined after
+ * T == 0 or I == 0 is valid: only zero_count (= 0) is written.
+ */
+int cq_quantize_act(const void* X, int dtype, int64_t T, int64_t I, int64_t ld,
+                    double alpha, int bits,
+                    float* t, float* c, float* row_scale, float* col_scale,
+                    void* codes, void* deq, int deq_dtype,
+                    unsigned long long* zero_count,
+                    void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Same operation on HOST buffers: copies X to the device, runs cq_quantize_act and copies
+ * every requested output back, all on `stream`.  Host pointers should be page-locked for the
+ * copies to be asynchronous.  `device_scratch` (device, 256-byte aligned) must hold
+ * cq_host_scratch_bytes(...) bytes.  Outputs are complete once `stream` has been synchronised
+ * by the caller.  zero_count is a HOST uint64 here.
+ */
+size_t cq_host_scratch_bytes(int64_t T, int64_t I, int bits, int want_codes, int want_deq, int deq_dtype);
+int cq_quantize_act_host(const void* X_host, int dtype, int64_t T, int64_t I, int64_t ld,
+                         double alpha, int bits,
+                         float* t_host, float* c_host, float* row_scale_host, float* col_scale_host,
+                         void* codes_host, void* deq_host, int deq_dtype,
+                         unsigned long long* zero_count_host,
+                         void* device_scratch, size_t scratch_bytes, void* stream);
+
+/* xhat_ij = fl32(code_ij * fl32(row_scale_i * col_scale_j)) from stored codes (the last step of
+ * the Appendix B.1 listing).  out: device [T*I] of out_dtype (CQ_F16, CQ_BF16 or CQ_F32). */
+int cq_dequantize(const void* codes, int bits, int64_t T, int64_t I,
+                  const float* row_scale, const float* col_scale,
+                  void* out, int out_dtype, void* stream);
+
+/* |K| = number of zero codes (Definition 1) in stored codes.  count: device uint64. */
+int cq_kernel_count(const void* codes, int bits, int64_t T, int64_t I,
+                    unsigned long long* count, void* stream);
+
+/* |K(CQ)| straight from X, without storing codes (the kernel-proportion analysis of
+ * Section 4.2).  t, c: device, as produced by cq_absmax_rows_cols on the same X. */
+int cq_kernel_count_x(const void* X, int dtype, int64_t T, int64_t I, int64_t ld,
+                      double alpha, int bits, const float* t, const float* c,
+                      unsigned long long* count,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Per-channel weight quantization (Eq. 2): one scale per STORED row r,
+ *   d_r = fl32(max_k |W_rk| / qmax), code = round-half-even(fl32(W_rk / d_r)), what = fl32(code * d_r).
+ * Store weights as [output channels x input channels] to get one scale per output channel.
+ *   W in device [R x ld]; codes out int8[R*C] or packed uint8[R*C/2]; scale out float[R];
+ *   deq out [R*C] of deq_dtype (W's dtype or CQ_F32); zero_count out device uint64.
+ *   codes, scale, deq, zero_count are nullable.  Each row is read from HBM once while it fits
+ *   in shared memory (C <= 110,592), twice otherwise.
+ */
+int cq_quantize_weight_per_channel(const void* W, int dtype, int64_t R, int64_t C, int64_t ld, int bits,
+                                   void* codes, float* scale, void* deq, int deq_dtype,
+                                   unsigned long long* zero_count, void* stream);
+
+/* Launch-shape knobs for measurement (rows per CTA of the two passes, CTAs per SM hints).
+ * key: "k1_rows", "k3_rows".  value <= 0 restores the built-in choice.  Returns CQ_OK or CQ_ERR_SHAPE. */
+int cq_set_tuning(const char* key, int value);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CQ_H_ */

@@ -1,0 +1,295 @@
+"""Thin binding of the C-ABI library ``libcq.so`` (argument marshalling only).
+
+Every function has the name of the C entry point without the ``cq_`` prefix and does no
+arithmetic of its own: torch supplies device memory and the current stream, ctypes passes raw
+pointers.  A missing or unloadable library is an error -- there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libcq.so")
+
+CQ_F16, CQ_BF16, CQ_F32 = 0, 1, 2
+_DT = {torch.float16: CQ_F16, torch.bfloat16: CQ_BF16, torch.float32: CQ_F32}
+
+EXPORTS = (
+    "cq_version", "cq_status_string", "cq_absmax_rows", "cq_absmax_cols", "cq_absmax_rows_cols",
+    "cq_workspace_bytes", "cq_quantize_act", "cq_host_scratch_bytes", "cq_quantize_act_host",
+    "cq_dequantize", "cq_kernel_count", "cq_kernel_count_x", "cq_quantize_weight_per_channel",
+    "cq_set_tuning",
+)
+
+
+class CQError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: status {status} ({status_string(status)})")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load libcq.so (built by ``paper_2410_07505_b200.build``); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} not found: build it with `python -m paper_2410_07505_b200.build`")
+        L = C.CDLL(LIB_PATH)
+        i64, vp, dbl, ci = C.c_int64, C.c_void_p, C.c_double, C.c_int
+        L.cq_version.restype = ci
+        L.cq_status_string.restype = C.c_char_p
+        L.cq_status_string.argtypes = [ci]
+        L.cq_absmax_rows.argtypes = [vp, ci, i64, i64, i64, vp, vp]
+        L.cq_absmax_cols.argtypes = [vp, ci, i64, i64, i64, vp, vp]
+        L.cq_absmax_rows_cols.argtypes = [vp, ci, i64, i64, i64, vp, vp, vp]
+        L.cq_workspace_bytes.restype = C.c_size_t
+        L.cq_workspace_bytes.argtypes = [i64, i64]
+        L.cq_quantize_act.argtypes = [vp, ci, i64, i64, i64, dbl, ci, vp, vp, vp, vp, vp, vp, ci, vp, vp,
+                                      C.c_size_t, vp]
+        L.cq_host_scratch_bytes.restype = C.c_size_t
+        L.cq_host_scratch_bytes.argtypes = [i64, i64, ci, ci, ci, ci]
+        L.cq_quantize_act_host.argtypes = [vp, ci, i64, i64, i64, dbl, ci, vp, vp, vp, vp, vp, vp, ci, vp, vp,
+                                           C.c_size_t, vp]
+        L.cq_dequantize.argtypes = [vp, ci, i64, i64, vp, vp, vp, ci, vp]
+        L.cq_kernel_count.argtypes = [vp, ci, i64, i64, vp, vp]
+        L.cq_kernel_count_x.argtypes = [vp, ci, i64, i64, i64, dbl, ci, vp, vp, vp, vp, C.c_size_t, vp]
+        L.cq_quantize_weight_per_channel.argtypes = [vp, ci, i64, i64, i64, ci, vp, vp, vp, ci, vp, vp]
+        L.cq_set_tuning.argtypes = [C.c_char_p, ci]
+        for name in EXPORTS:
+            if name not in ("cq_status_string", "cq_workspace_bytes", "cq_host_scratch_bytes"):
+                getattr(L, name).restype = ci
+        _lib = L
+    return _lib
+
+
+def version() -> int:
+    return int(lib().cq_version())
+
+
+def status_string(status: int) -> str:
+    return lib().cq_status_string(int(status)).decode()
+
+
+def set_tuning(key: str, value: int) -> None:
+    _check(lib().cq_set_tuning(key.encode(), int(value)), "cq_set_tuning")
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise CQError(status, where)
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _matrix_args(X: torch.Tensor):
+    if X.dim() != 2 or X.dtype not in (torch.float16, torch.bfloat16):
+        raise TypeError("expected a 2-D float16 / bfloat16 tensor")
+    if not X.is_cuda:
+        raise TypeError("expected a CUDA tensor")
+    T, I = X.shape
+    if I > 0 and T > 0 and X.stride(1) != 1:
+        raise ValueError("columns must be contiguous")
+    ld = X.stride(0) if T > 1 else max(I, 1)
+    return T, I, ld
+
+
+def workspace_bytes(T: int, I: int) -> int:
+    return int(lib().cq_workspace_bytes(T, I))
+
+
+def _workspace(T, I, device):
+    return torch.empty(workspace_bytes(T, I), dtype=torch.uint8, device=device)
+
+
+# ----------------------------------------------------------------------------- absmax
+def absmax_rows(X: torch.Tensor) -> torch.Tensor:
+    T, I, ld = _matrix_args(X)
+    t = torch.empty(T, dtype=torch.float32, device=X.device)
+    _check(lib().cq_absmax_rows(_ptr(X), _DT[X.dtype], T, I, ld, _ptr(t), _stream()), "cq_absmax_rows")
+    return t
+
+
+def absmax_cols(X: torch.Tensor) -> torch.Tensor:
+    T, I, ld = _matrix_args(X)
+    c = torch.empty(I, dtype=torch.float32, device=X.device)
+    _check(lib().cq_absmax_cols(_ptr(X), _DT[X.dtype], T, I, ld, _ptr(c), _stream()), "cq_absmax_cols")
+    return c
+
+
+def absmax_rows_cols(X: torch.Tensor):
+    T, I, ld = _matrix_args(X)
+    t = torch.empty(T, dtype=torch.float32, device=X.device)
+    c = torch.empty(I, dtype=torch.float32, device=X.device)
+    _check(lib().cq_absmax_rows_cols(_ptr(X), _DT[X.dtype], T, I, ld, _ptr(t), _ptr(c), _stream()),
+           "cq_absmax_rows_cols")
+    return t, c
+
+
+# ----------------------------------------------------------------------------- quantize
+@dataclass
+class ActQuant:
+    t: torch.Tensor | None
+    c: torch.Tensor | None
+    row_scale: torch.Tensor | None
+    col_scale: torch.Tensor | None
+    codes: torch.Tensor | None        # int8 [T, I] or uint8 [T, I/2]
+    deq: torch.Tensor | None
+    zero_count: torch.Tensor | None   # uint64 scalar stored as int64 on the device
+    bits: int
+
+    def kernel_proportion(self) -> float:
+        n = self.t.numel() * self.c.numel()
+        return int(self.zero_count.item()) / n if n else 0.0
+
+
+class ActBuffers:
+    """Pre-allocated outputs and workspace for repeated calls on one shape."""
+
+    def __init__(self, T, I, dtype, bits, *, codes=True, deq=True, deq_dtype=None, count=True, device="cuda"):
+        dev = torch.device(device)
+        self.T, self.I, self.bits = T, I, bits
+        self.t = torch.empty(T, dtype=torch.float32, device=dev)
+        self.c = torch.empty(I, dtype=torch.float32, device=dev)
+        self.row_scale = torch.empty(T, dtype=torch.float32, device=dev)
+        self.col_scale = torch.empty(I, dtype=torch.float32, device=dev)
+        self.codes = None
+        if codes:
+            self.codes = (torch.empty((T, I), dtype=torch.int8, device=dev) if bits == 8
+                          else torch.empty((T, I // 2), dtype=torch.uint8, device=dev))
+        self.deq = torch.empty((T, I), dtype=deq_dtype or dtype, device=dev) if deq else None
+        self.zero_count = torch.zeros((), dtype=torch.int64, device=dev) if count else None
+        self.workspace = _workspace(T, I, dev)
+
+
+def quantize_act(X: torch.Tensor, alpha: float = 0.15, bits: int = 8, *, codes: bool = True,
+                 deq: bool = True, deq_dtype: torch.dtype | None = None, count: bool = True,
+                 buffers: ActBuffers | None = None) -> ActQuant:
+    """CrossQuant of X (tokens x channels): t, c, scale vectors, codes, dequantized X, |K(CQ)|."""
+    T, I, ld = _matrix_args(X)
+    if bits == 4 and I % 2:
+        raise CQError(6, "cq_quantize_act")
+    b = buffers or ActBuffers(T, I, X.dtype, bits, codes=codes, deq=deq, deq_dtype=deq_dtype, count=count,
+                              device=X.device)
+    deq_dt = _DT[b.deq.dtype] if b.deq is not None else _DT[X.dtype]
+    st = lib().cq_quantize_act(_ptr(X), _DT[X.dtype], T, I, ld, float(alpha), int(bits), _ptr(b.t), _ptr(b.c),
+                               _ptr(b.row_scale), _ptr(b.col_scale), _ptr(b.codes), _ptr(b.deq), deq_dt,
+                               _ptr(b.zero_count), _ptr(b.workspace), b.workspace.numel(), _stream())
+    _check(st, "cq_quantize_act")
+    return ActQuant(b.t, b.c, b.row_scale, b.col_scale, b.codes, b.deq, b.zero_count, bits)
+
+
+class HostBuffers:
+    """Page-locked host outputs plus the device scratch of the host-buffer entry point."""
+
+    def __init__(self, T, I, dtype, bits, *, codes=True, deq=True, deq_dtype=None, device="cuda"):
+        self.T, self.I, self.bits = T, I, bits
+        pin = dict(pin_memory=True)
+        self.t = torch.empty(T, dtype=torch.float32, **pin)
+        self.c = torch.empty(I, dtype=torch.float32, **pin)
+        self.row_scale = torch.empty(T, dtype=torch.float32, **pin)
+        self.col_scale = torch.empty(I, dtype=torch.float32, **pin)
+        self.codes = None
+        if codes:
+            self.codes = (torch.empty((T, I), dtype=torch.int8, **pin) if bits == 8
+                          else torch.empty((T, I // 2), dtype=torch.uint8, **pin))
+        self.deq = torch.empty((T, I), dtype=deq_dtype or dtype, **pin) if deq else None
+        self.zero_count = torch.zeros((), dtype=torch.int64, **pin)
+        deq_dt = _DT[self.deq.dtype] if self.deq is not None else _DT[dtype]
+        n = int(lib().cq_host_scratch_bytes(T, I, bits, int(codes), int(deq), deq_dt))
+        self.scratch = torch.empty(n, dtype=torch.uint8, device=device)
+
+    def d2h_bytes(self) -> int:
+        n = 4 * (2 * self.T + 2 * self.I) + 8
+        for x in (self.codes, self.deq):
+            if x is not None:
+                n += x.numel() * x.element_size()
+        return n
+
+
+def quantize_act_host(X_host: torch.Tensor, alpha: float = 0.15, bits: int = 8, *,
+                      buffers: HostBuffers) -> ActQuant:
+    """Same as quantize_act on a HOST matrix; results land in ``buffers`` (host) once the current
+    stream has been synchronised."""
+    if X_host.is_cuda or X_host.dim() != 2 or X_host.dtype not in (torch.float16, torch.bfloat16):
+        raise TypeError("expected a 2-D float16 / bfloat16 host tensor")
+    T, I = X_host.shape
+    ld = X_host.stride(0) if T > 1 else max(I, 1)
+    b = buffers
+    deq_dt = _DT[b.deq.dtype] if b.deq is not None else _DT[X_host.dtype]
+    st = lib().cq_quantize_act_host(_ptr(X_host), _DT[X_host.dtype], T, I, ld, float(alpha), int(bits),
+                                    _ptr(b.t), _ptr(b.c), _ptr(b.row_scale), _ptr(b.col_scale), _ptr(b.codes),
+                                    _ptr(b.deq), deq_dt, _ptr(b.zero_count), _ptr(b.scratch), b.scratch.numel(),
+                                    _stream())
+    _check(st, "cq_quantize_act_host")
+    return ActQuant(b.t, b.c, b.row_scale, b.col_scale, b.codes, b.deq, b.zero_count, bits)
+
+
+def dequantize(codes: torch.Tensor, bits: int, T: int, I: int, row_scale: torch.Tensor, col_scale: torch.Tensor,
+               out_dtype: torch.dtype = torch.float32) -> torch.Tensor:
+    out = torch.empty((T, I), dtype=out_dtype, device=codes.device)
+    _check(lib().cq_dequantize(_ptr(codes), int(bits), T, I, _ptr(row_scale), _ptr(col_scale), _ptr(out),
+                               _DT[out_dtype], _stream()), "cq_dequantize")
+    return out
+
+
+def kernel_count(codes: torch.Tensor, bits: int, T: int, I: int) -> torch.Tensor:
+    count = torch.zeros((), dtype=torch.int64, device=codes.device)
+    _check(lib().cq_kernel_count(_ptr(codes), int(bits), T, I, _ptr(count), _stream()), "cq_kernel_count")
+    return count
+
+
+def kernel_count_x(X: torch.Tensor, alpha: float, bits: int, t: torch.Tensor, c: torch.Tensor,
+                   workspace: torch.Tensor | None = None) -> torch.Tensor:
+    T, I, ld = _matrix_args(X)
+    ws = workspace if workspace is not None else _workspace(T, I, X.device)
+    count = torch.zeros((), dtype=torch.int64, device=X.device)
+    _check(lib().cq_kernel_count_x(_ptr(X), _DT[X.dtype], T, I, ld, float(alpha), int(bits), _ptr(t), _ptr(c),
+                                   _ptr(count), _ptr(ws), ws.numel(), _stream()), "cq_kernel_count_x")
+    return count
+
+
+@dataclass
+class WeightQuant:
+    scale: torch.Tensor
+    codes: torch.Tensor | None
+    deq: torch.Tensor | None
+    zero_count: torch.Tensor | None
+    bits: int
+
+
+def quantize_weight_per_channel(W: torch.Tensor, bits: int = 8, *, codes: bool = True, deq: bool = True,
+                                deq_dtype: torch.dtype | None = None, count: bool = True,
+                                out: WeightQuant | None = None) -> WeightQuant:
+    """Eq. 2: one scale per stored row of W (store weights as [out_channels, in_channels])."""
+    R, Cc, ld = _matrix_args(W)
+    if bits == 4 and Cc % 2:
+        raise CQError(6, "cq_quantize_weight_per_channel")
+    if out is None:
+        dev = W.device
+        codes_t = None
+        if codes:
+            codes_t = (torch.empty((R, Cc), dtype=torch.int8, device=dev) if bits == 8
+                       else torch.empty((R, Cc // 2), dtype=torch.uint8, device=dev))
+        out = WeightQuant(torch.empty(R, dtype=torch.float32, device=dev), codes_t,
+                          torch.empty((R, Cc), dtype=deq_dtype or W.dtype, device=dev) if deq else None,
+                          torch.zeros((), dtype=torch.int64, device=dev) if count else None, bits)
+    deq_dt = _DT[out.deq.dtype] if out.deq is not None else _DT[W.dtype]
+    st = lib().cq_quantize_weight_per_channel(_ptr(W), _DT[W.dtype], R, Cc, ld, int(bits), _ptr(out.codes),
+                                              _ptr(out.scale), _ptr(out.deq), deq_dt, _ptr(out.zero_count),
+                                              _stream())
+    _check(st, "cq_quantize_weight_per_channel")
+    return out

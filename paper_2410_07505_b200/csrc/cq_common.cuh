@@ -1,0 +1,153 @@
+// Device-side helpers shared by the CrossQuant kernels (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "cq.h"
+
+namespace cq {
+
+// Adding 1.5 * 2^23 to a float of magnitude < 2^22 leaves round-half-even(v) in the low mantissa
+// bits: bits(v + kMagic) == kMagicBits + rint(v) as a two's-complement integer.
+constexpr float kMagic = 12582912.0f;
+constexpr uint32_t kMagicBits = 0x4B400000u;
+// 1/2 - 2^-16: a candidate code q is accepted without the IEEE division when |x - q s| < s * kHalfMinus.
+constexpr float kHalfMinus = 0.4999847412109375f;
+
+constexpr int kThreads = 256;      // largest CTA of the tiled kernels
+constexpr int kMaxRowsPerCta = 128;
+
+__device__ __forceinline__ uint32_t max_u16x2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("max.u16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+
+__device__ __forceinline__ uint4 ld_nc(const uint4* p) { return __ldg(p); }
+
+// streaming (evict-first) accesses for data touched once
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) { return __ldcs(p); }
+__device__ __forceinline__ void st_stream(uint4* p, uint4 v) { __stcs(p, v); }
+__device__ __forceinline__ void st_stream(uint2* p, uint2 v) { __stcs(p, v); }
+__device__ __forceinline__ void st_stream(uint32_t* p, uint32_t v) { __stcs(p, v); }
+__device__ __forceinline__ void st_stream(float4* p, float4 v) { __stcs(p, v); }
+
+// ---- 16-bit formats ------------------------------------------------------------------------
+template <int DT>
+__device__ __forceinline__ float2 unpack16x2(uint32_t w) {
+    if constexpr (DT == CQ_BF16) {
+        return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u));
+    } else {
+        __half2 h = *reinterpret_cast<__half2*>(&w);
+        return __half22float2(h);
+    }
+}
+
+template <int DT>
+__device__ __forceinline__ float cvt16(uint16_t bits) {
+    if constexpr (DT == CQ_BF16) {
+        return __uint_as_float(static_cast<uint32_t>(bits) << 16);
+    } else {
+        return __half2float(__ushort_as_half(bits));
+    }
+}
+
+__device__ __forceinline__ float cvt16_rt(uint16_t bits, int dt) {
+    return dt == CQ_BF16 ? cvt16<CQ_BF16>(bits) : cvt16<CQ_F16>(bits);
+}
+
+// two floats -> packed 16-bit pair, round to nearest even
+template <int DT>
+__device__ __forceinline__ uint32_t pack16x2(float lo, float hi) {
+    if constexpr (DT == CQ_BF16) {
+        __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+        return *reinterpret_cast<uint32_t*>(&p);
+    } else {
+        __half2 p = __floats2half2_rn(lo, hi);
+        return *reinterpret_cast<uint32_t*>(&p);
+    }
+}
+
+template <int DT>
+__device__ __forceinline__ uint16_t pack16(float v) {
+    if constexpr (DT == CQ_BF16) {
+        return __bfloat16_as_ushort(__float2bfloat16_rn(v));
+    } else {
+        return __half_as_ushort(__float2half_rn(v));
+    }
+}
+
+// ---- one element ---------------------------------------------------------------------------
+// Candidate code from a reciprocal product; returns kMagic + q.  `ok` tells whether q is proven
+// equal to round-half-even(fl32(x / s)): with z = x/s and |z| <= 128, fl32(z) lies within 2^-17 of
+// z, so |z - q| < 1/2 - 2^-16 (checked on the exactly computed residual x - q s) forces the IEEE
+// quotient to round to q as well.  Any NaN or infinity in the candidate makes the test fail.
+__device__ __forceinline__ float quant_candidate(float x, float s, float r, float qmaxf, bool& ok) {
+    float v = __fmul_rn(x, r);
+    v = fminf(fmaxf(v, -qmaxf), qmaxf);
+    float y = __fadd_rn(v, kMagic);
+    float qf = __fadd_rn(y, -kMagic);
+    float e = __fmaf_rn(-qf, s, x);
+    ok = fabsf(e) < __fmul_rn(s, kHalfMinus);
+    return y;
+}
+
+// The defining sequence: IEEE division, round half to even, clamp.  Returns kMagic + q.
+static __device__ __noinline__ float quant_exact(float x, float s, float qmaxf) {
+    if (s == 0.0f) return kMagic;
+    float u = __fdiv_rn(x, s);
+    float q = rintf(u);
+    q = fminf(fmaxf(q, -qmaxf), qmaxf);
+    return __fadd_rn(q, kMagic);        // (-0) + kMagic == kMagic
+}
+
+__device__ __forceinline__ float code_as_float(float y) { return __fadd_rn(y, -kMagic); }
+__device__ __forceinline__ int code_as_int(float y) {
+    return static_cast<int>(__float_as_uint(y)) - static_cast<int>(kMagicBits);
+}
+
+// four codes (low bytes of four magic-biased floats) -> one word of int8
+__device__ __forceinline__ uint32_t pack_int8x4(float y0, float y1, float y2, float y3) {
+    uint32_t p01 = __byte_perm(__float_as_uint(y0), __float_as_uint(y1), 0x0040);
+    uint32_t p23 = __byte_perm(__float_as_uint(y2), __float_as_uint(y3), 0x0040);
+    return __byte_perm(p01, p23, 0x5410);
+}
+
+// eight codes -> one word of two's-complement nibbles, element e in bits [4e, 4e+4)
+__device__ __forceinline__ uint32_t pack_int4x8(const float (&y)[8]) {
+    uint32_t w = 0;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) w |= (__float_as_uint(y[e]) & 0xFu) << (4 * e);
+    return w;
+}
+
+__device__ __forceinline__ int zero_bytes(uint32_t w) {
+    uint32_t t = (w & 0x7F7F7F7Fu) + 0x7F7F7F7Fu;
+    t = ~(t | w | 0x7F7F7F7Fu);
+    return __popc(t);
+}
+
+__device__ __forceinline__ int zero_nibbles(uint32_t w) {
+    uint32_t nz = (w | (w >> 1) | (w >> 2) | (w >> 3)) & 0x11111111u;
+    return 8 - __popc(nz);
+}
+
+// CTA-wide sum of per-thread counts, one atomic per CTA
+__device__ __forceinline__ void cta_count_add(unsigned int cnt, unsigned long long* dst) {
+    __shared__ unsigned int s_cnt[kThreads / 32];
+    unsigned int w = __reduce_add_sync(0xFFFFFFFFu, cnt);
+    int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) s_cnt[warp] = w;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned long long sum = 0;
+        int nw = (blockDim.x + 31) >> 5;
+        for (int k = 0; k < nw; ++k) sum += s_cnt[k];
+        if (sum) atomicAdd(dst, sum);
+    }
+}
+
+}  // namespace cq

@@ -1,0 +1,28 @@
+// Host-side declarations shared by the translation units of libcq.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace cq {
+
+// Tiling of a T x I matrix and the carving of the caller's workspace.
+struct Plan {
+    int I8;        // vectors of 8 columns per row
+    int W;         // threads per CTA = vectors per column strip
+    int nstrips;   // column strips
+    int R1, nrb1;  // rows per CTA and row blocks of the absmax pass
+    int R3, nrb3;  // the same for the quantize pass
+    size_t off_t, off_c, off_a, off_b, off_ra, off_rb, off_rowpart, off_colpart, total;
+};
+
+Plan make_plan(int64_t T, int64_t I);
+int check_matrix(const void* X, int dtype, int64_t T, int64_t I, int64_t ld);
+int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld, double alpha, int bits,
+                      const float* t_given, const float* c_given,
+                      float* t, float* c, float* row_scale, float* col_scale,
+                      void* codes, void* deq, int deq_dtype, unsigned long long* zero_count,
+                      void* workspace, size_t ws_bytes, cudaStream_t st);
+
+}  // namespace cq

@@ -1,0 +1,268 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import cq_oracle as orc
+from oracle import parity
+from paper_2410_07505_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+TORCH_DT = {"f16": torch.float16, "bf16": torch.bfloat16}
+
+
+@pytest.fixture(scope="module")
+def cq():
+    if not torch.cuda.is_available():
+        pytest.fail("the gpu tests need a CUDA device")
+    from paper_2410_07505_b200 import build, cq as _cq
+    build.build()
+    _cq.lib()
+    return _cq
+
+
+def to_dev(bits: np.ndarray, dtype: str) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(TORCH_DT[dtype]).cuda()
+
+
+def bits_of(t: torch.Tensor) -> np.ndarray:
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def run_and_check(cq, X, dtype, alpha, bits, *, deq_f32=False, Xd=None, ref=None):
+    Xd = to_dev(X, dtype) if Xd is None else Xd
+    r = cq.quantize_act(Xd, alpha, bits, deq_dtype=torch.float32 if deq_f32 else None)
+    torch.cuda.synchronize()
+    deq = r.deq.cpu().numpy() if deq_f32 else bits_of(r.deq)
+    return parity.check_act(X, dtype, alpha, bits, t=r.t.cpu().numpy(), c=r.c.cpu().numpy(),
+                            a=r.row_scale.cpu().numpy(), b=r.col_scale.cpu().numpy(),
+                            codes=r.codes.cpu().numpy(), deq=deq, deq_is_f32=deq_f32,
+                            zero_count=int(r.zero_count.item()), ref=ref), r
+
+
+# ------------------------------------------------------------------ small, multi-tile, ragged
+FAST_SHAPES = [(1, 8), (3, 16), (37, 264), (130, 2056), (257, 776), (64, 4104), (19, 2048)]
+GENERAL_SHAPES = [(1, 1), (5, 7), (33, 50), (17, 1001), (70, 258)]
+
+
+@pytest.mark.parametrize("shape", FAST_SHAPES + GENERAL_SHAPES)
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+def test_small_shapes_all_alphas_and_bit_widths(cq, shape, dtype):
+    T, I = shape
+    X = wl.small_matrix(T, I, dtype, 1000 + T + I, outlier_cols=2, zero_frac=0.01)
+    for bits in (8, 4):
+        if bits == 4 and I % 2:
+            continue
+        for alpha in (0.0, 0.15, 0.5, 1.0):
+            rep, _ = run_and_check(cq, X, dtype, alpha, bits)
+            assert rep.scales_identical and rep.code_mismatches == 0
+    rep, _ = run_and_check(cq, X, dtype, 0.15, 8, deq_f32=True)
+    assert rep.max_deq_ulp == 0
+
+
+@pytest.mark.parametrize("dist", ["student_t3", "laplace"])
+def test_heavy_tailed_values(cq, dist):
+    X = wl.small_matrix(300, 1536, "bf16", 77, dist=dist, outlier_cols=5, outlier_scale=50.0)
+    for alpha in (0.15, 0.45, 0.75):
+        for bits in (8, 4):
+            run_and_check(cq, X, "bf16", alpha, bits)
+
+
+def test_leading_dimension_and_offset_views(cq):
+    big = wl.small_matrix(90, 640, "bf16", 5)
+    bd = to_dev(big, "bf16")
+    # aligned window: fast kernels with ld > I
+    win = np.ascontiguousarray(big[:, 64:64 + 256])
+    run_and_check(cq, win, "bf16", 0.15, 8, Xd=bd[:, 64:64 + 256])
+    run_and_check(cq, win, "bf16", 0.5, 4, Xd=bd[:, 64:64 + 256])
+    # odd offset: pointer only 2-byte aligned -> general kernels
+    win = np.ascontiguousarray(big[:, 3:3 + 250])
+    run_and_check(cq, win, "bf16", 0.15, 8, Xd=bd[:, 3:3 + 250])
+    run_and_check(cq, win, "bf16", 0.15, 4, Xd=bd[:, 3:3 + 250])
+
+
+def test_empty_matrices(cq):
+    for T, I in [(0, 64), (16, 0), (0, 0)]:
+        Xd = torch.empty((T, I), dtype=torch.float16, device="cuda")
+        r = cq.quantize_act(Xd, 0.15, 8)
+        torch.cuda.synchronize()
+        assert int(r.zero_count.item()) == 0
+        assert cq.absmax_rows(Xd).shape == (T,) and cq.absmax_cols(Xd).shape == (I,)
+        if T == 0 and I > 0:
+            assert not cq.absmax_cols(Xd).any()
+
+
+@pytest.mark.parametrize("alpha", [0.0, 0.15, 1.0])
+def test_zero_row_zero_column_and_all_zero(cq, alpha):
+    X = wl.small_matrix(40, 128, "bf16", 9, outlier_cols=0)
+    X[7, :] = 0
+    X[:, 11] = 0x8000
+    rep, r = run_and_check(cq, X, "bf16", alpha, 8, deq_f32=True)
+    assert torch.isfinite(r.deq).all()
+    assert not r.codes[7].any() and not r.codes[:, 11].any()
+    Z = np.zeros((16, 64), dtype=np.uint16)
+    rep, r = run_and_check(cq, Z, "f16", alpha, 4)
+    assert rep.zero_count == 16 * 64
+
+
+def test_extreme_magnitudes(cq):
+    # largest fp16 values
+    X = wl.small_matrix(32, 256, "f16", 3, scale=3000.0, outlier_cols=2, outlier_scale=20.0)
+    X[0, 0] = 0x7BFF
+    X[5, 9] = 0xFBFF
+    run_and_check(cq, X, "f16", 0.15, 8)
+    run_and_check(cq, X, "f16", 0.15, 8, deq_f32=True)
+    # fp16 subnormals only
+    S = (np.arange(32 * 64, dtype=np.uint16).reshape(32, 64) % 1024)
+    S[1::2] |= 0x8000
+    run_and_check(cq, S, "f16", 0.5, 8)
+    # bf16 near the top and the bottom of the fp32 exponent range (scales become subnormal)
+    for scale in (1e36, 1e-36, 3e-39):
+        B = wl.small_matrix(24, 128, "bf16", 4, scale=scale, outlier_cols=1, outlier_scale=8.0)
+        for alpha in (0.0, 0.15, 0.5, 1.0):
+            run_and_check(cq, B, "bf16", alpha, 8, deq_f32=True)
+            run_and_check(cq, B, "bf16", alpha, 4)
+
+
+def test_exact_ties_round_to_even_on_the_gpu(cq):
+    row = np.zeros((1, 16), dtype=np.float32)
+    row[0, :10] = [127, 0.5, 1.5, 2.5, -0.5, -1.5, -2.5, 3.5, 126.5, -125.5]
+    X = wl.to_bits(row, "f16")
+    rep, r = run_and_check(cq, X, "f16", 1.0, 8)
+    assert r.codes[0, :10].tolist() == [127, 0, 2, 2, 0, -2, -2, 4, 126, -126]
+
+
+def test_outputs_are_optional(cq):
+    X = wl.small_matrix(65, 512, "bf16", 12)
+    Xd = to_dev(X, "bf16")
+    ref = orc.quantize_act(X, "bf16", 0.15, 8)
+    r = cq.quantize_act(Xd, 0.15, 8, codes=False, deq=False)
+    assert int(r.zero_count.item()) == ref.zero_count
+    r = cq.quantize_act(Xd, 0.15, 8, codes=True, deq=False, count=False)
+    assert np.array_equal(r.codes.cpu().numpy(), ref.codes)
+    r = cq.quantize_act(Xd, 0.15, 8, codes=False, deq=True, count=False)
+    assert np.array_equal(bits_of(r.deq), ref.deq16)
+
+
+def test_tiling_knobs_do_not_change_results(cq):
+    X = wl.small_matrix(333, 2304, "bf16", 13, outlier_cols=3)
+    ref = orc.quantize_act(X, "bf16", 0.15, 8)
+    try:
+        for k1, k3 in [(16, 4), (32, 64), (128, 128), (64, 8)]:
+            cq.set_tuning("k1_rows", k1)
+            cq.set_tuning("k3_rows", k3)
+            run_and_check(cq, X, "bf16", 0.15, 8, ref=ref)
+    finally:
+        cq.set_tuning("k1_rows", 0)
+        cq.set_tuning("k3_rows", 0)
+
+
+def test_repeated_calls_reuse_buffers(cq):
+    X = wl.small_matrix(128, 1024, "f16", 14)
+    Xd = to_dev(X, "f16")
+    buf = cq.ActBuffers(128, 1024, torch.float16, 8)
+    ref = orc.quantize_act(X, "f16", 0.15, 8)
+    for _ in range(3):
+        r = cq.quantize_act(Xd, 0.15, 8, buffers=buf)
+        assert int(r.zero_count.item()) == ref.zero_count
+        assert np.array_equal(r.codes.cpu().numpy(), ref.codes)
+
+
+# ------------------------------------------------------------------ the other entry points
+@pytest.mark.parametrize("shape,dtype", [((130, 2056), "bf16"), ((33, 50), "f16"), ((1, 8), "f16"), ((700, 96), "bf16")])
+def test_absmax_entry_points(cq, shape, dtype):
+    X = wl.small_matrix(*shape, dtype, 21)
+    Xd = to_dev(X, dtype)
+    t_ref, c_ref = orc.absmax_rows(X, dtype), orc.absmax_cols(X, dtype)
+    t, c = cq.absmax_rows_cols(Xd)
+    assert np.array_equal(t.cpu().numpy(), t_ref) and np.array_equal(c.cpu().numpy(), c_ref)
+    assert np.array_equal(cq.absmax_rows(Xd).cpu().numpy(), t_ref)
+    assert np.array_equal(cq.absmax_cols(Xd).cpu().numpy(), c_ref)
+
+
+@pytest.mark.parametrize("shape", [(65, 512), (33, 50), (9, 1030)])
+@pytest.mark.parametrize("bits", [8, 4])
+def test_dequantize_and_kernel_count_from_stored_codes(cq, shape, bits):
+    T, I = shape
+    X = wl.small_matrix(T, I, "bf16", 31, zero_frac=0.02)
+    ref = orc.quantize_act(X, "bf16", 0.15, bits)
+    stored = ref.codes if bits == 8 else ref.packed_int4()
+    cd = torch.from_numpy(stored).cuda()
+    a, b = torch.from_numpy(ref.a).cuda(), torch.from_numpy(ref.b).cuda()
+    out32 = cq.dequantize(cd, bits, T, I, a, b, torch.float32).cpu().numpy()
+    assert np.array_equal(out32.view(np.uint32), ref.deq32.view(np.uint32))
+    out16 = cq.dequantize(cd, bits, T, I, a, b, torch.bfloat16)
+    assert np.array_equal(bits_of(out16), ref.deq16)
+    outh = cq.dequantize(cd, bits, T, I, a, b, torch.float16)
+    assert np.array_equal(bits_of(outh), orc.encode16(ref.deq32, "f16"))
+    assert int(cq.kernel_count(cd, bits, T, I).item()) == ref.zero_count
+    # misaligned start of the code buffer
+    if bits == 8:
+        pad = torch.zeros(stored.size + 3, dtype=torch.int8, device="cuda")
+        pad[3:] = cd.flatten()
+        assert int(cq.kernel_count(pad[3:], bits, T, I).item()) == ref.zero_count
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+def test_kernel_count_straight_from_x(cq, bits):
+    X = wl.small_matrix(200, 1032, "f16", 41, outlier_cols=4, outlier_scale=40.0, zero_frac=0.01)
+    Xd = to_dev(X, "f16")
+    t, c = cq.absmax_rows_cols(Xd)
+    for alpha in (0.15, 1.0):
+        ref = orc.quantize_act(X, "f16", alpha, bits, want_deq32=False, want_deq16=False)
+        assert int(cq.kernel_count_x(Xd, alpha, bits, t, c).item()) == ref.zero_count
+
+
+WEIGHT_SHAPES = [(1, 8), (5, 264), (40, 2056), (7, 8192), (3, 28672), (33, 50), (6, 1001), (2, 110600)]
+
+
+@pytest.mark.parametrize("shape", WEIGHT_SHAPES)
+@pytest.mark.parametrize("bits", [8, 4])
+def test_weight_per_channel(cq, shape, bits):
+    R, Cc = shape
+    if bits == 4 and Cc % 2:
+        pytest.skip("INT4 needs an even number of columns")
+    for dtype in ("bf16", "f16"):
+        W = wl.small_matrix(R, Cc, dtype, 51 + R, scale=0.02, outlier_cols=1, outlier_scale=6.0)
+        if R > 2:
+            W[1, :] = 0
+        Wd = to_dev(W, dtype)
+        ref = orc.quantize_weight_per_channel(W, dtype, bits)
+        r = cq.quantize_weight_per_channel(Wd, bits)
+        torch.cuda.synchronize()
+        parity.check_weight(W, dtype, bits, scale=r.scale.cpu().numpy(), codes=r.codes.cpu().numpy(),
+                            deq=bits_of(r.deq), zero_count=int(r.zero_count.item()), ref=ref)
+        r = cq.quantize_weight_per_channel(Wd, bits, deq_dtype=torch.float32)
+        parity.check_weight(W, dtype, bits, deq=r.deq.cpu().numpy(), deq_is_f32=True, ref=ref)
+
+
+def test_weight_quantizer_equals_alpha_one_activation_path(cq):
+    W = wl.small_matrix(64, 1024, "bf16", 61, scale=0.02, outlier_cols=0)
+    Wd = to_dev(W, "bf16")
+    rw = cq.quantize_weight_per_channel(Wd, 8)
+    ra = cq.quantize_act(Wd, 1.0, 8)
+    assert torch.equal(rw.codes, ra.codes) and torch.equal(rw.scale, ra.row_scale)
+
+
+def test_host_buffer_entry_point(cq):
+    X = wl.small_matrix(300, 1536, "bf16", 71, outlier_cols=3)
+    Xh = torch.from_numpy(X.view(np.int16)).view(torch.bfloat16).pin_memory()
+    for bits in (8, 4):
+        buf = cq.HostBuffers(300, 1536, torch.bfloat16, bits)
+        r = cq.quantize_act_host(Xh, 0.15, bits, buffers=buf)
+        torch.cuda.synchronize()
+        parity.check_act(X, "bf16", 0.15, bits, t=r.t.numpy(), c=r.c.numpy(), a=r.row_scale.numpy(),
+                         b=r.col_scale.numpy(), codes=r.codes.numpy(),
+                         deq=r.deq.view(torch.int16).numpy().view(np.uint16), zero_count=int(r.zero_count.item()))
+
+
+def test_too_small_workspace_is_rejected_on_the_device(cq):
+    Xd = torch.zeros((64, 512), dtype=torch.float16, device="cuda")
+    buf = cq.ActBuffers(64, 512, torch.float16, 8)
+    buf.workspace = buf.workspace[:1024]
+    with pytest.raises(cq.CQError) as e:
+        cq.quantize_act(Xd, 0.15, 8, buffers=buf)
+    assert e.value.status == 7
