@@ -1,0 +1,303 @@
+#!/usr/bin/env python
+"""Benchmark of the CrossQuant activation quantizer on B200.
+
+One step = one full cq_quantize_act call (row/column absmax, scale vectors, INT8 codes, bf16
+dequantized matrix, zero-code count) on the LLaMA-70B-MLP-shaped activation matrix
+(4096 x 28672 bf16, Laplace values with 8 outlier channels x50, alpha = 0.15).  The metric is
+algorithmic bytes per second: 7 bytes per element (two compulsory reads of X, one byte of
+codes, two bytes of dequantized output) divided by the device time of the step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+With N > 1 (launched by torchrun, one rank per GPU) every rank quantizes its own matrix of the
+same shape: the path has no exchange step, so the ranks are independent (weak scaling).
+`--impl reference` times the CPU oracle, as it stands, on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "CrossQuant act-quant GB/s and % of HBM roofline at LLaMA-70B-shaped X"
+UNIT = "GB/s"
+ALPHA = 0.15
+BITS = 8
+BYTES_PER_ELEMENT_STEP = 7.0        # X read twice (2+2) + int8 codes (1) + bf16 dequantized (2)
+BYTES_PER_ELEMENT_QUANT_PASS = 5.0  # quantize pass alone: X (2) + codes (1) + dequantized (2)
+FALLBACK_HBM_GBS = 6650.0
+L2_FLUSH_BYTES = 256 << 20
+
+# DRAM traffic of the quantize pass from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum
+# per launch), valid only for the kernel sources whose digest is recorded with it.
+NCU_TRAFFIC = {"sources_sha256": None, "bytes_per_launch": None}
+
+
+def kernel_sources_digest() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for name in ("cq_act.cu", "cq_common.cuh"):
+        with open(os.path.join(ROOT, "paper_2410_07505_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, index: int, uuid: str | None = None, period_s: float = 0.02):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nvml = pynvml
+            try:
+                self.handle = pynvml.nvmlDeviceGetHandleByUUID(f"GPU-{uuid}".encode() if uuid else b"")
+            except Exception:
+                self.handle = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nvml = None
+
+    def _run(self):
+        n = self.nvml
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM)))
+                mask = int(n.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self.nvml is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": int(statistics.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def rank_config(rank: int):
+    from paper_2410_07505_b200 import workloads as wl
+    cfg = wl.ACT_CONFIGS[wl.HEADLINE]
+    if rank:
+        cfg = dataclasses.replace(cfg, seed=cfg.seed + 100 * rank)
+    return cfg
+
+
+def run_reference(args) -> None:
+    """The oracle, as it stands, on the host cores: each step is a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import cq_oracle as orc
+    from paper_2410_07505_b200 import workloads as wl
+    cfg = rank_config(0)
+    rows = 256
+    sample_cfg = dataclasses.replace(cfg, T=rows)
+    X = wl.generate_activation(sample_cfg)
+    for _ in range(args.warmup):
+        orc.quantize_act(X, cfg.dtype, ALPHA, BITS, want_deq32=False)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        orc.quantize_act(X, cfg.dtype, ALPHA, BITS, want_deq32=False)
+    dt = time.perf_counter() - t0
+    value = BYTES_PER_ELEMENT_STEP * X.size * args.steps / dt / 1e9
+    sample = f"first {rows} rows of the {cfg.T}x{cfg.I} matrix per step (oracle quantize_act: t, c, codes, bf16 dequant, count)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{cfg.name} {rows}x{cfg.I} bf16 sample, INT{BITS}, alpha={ALPHA}"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=10)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    from paper_2410_07505_b200 import build as cuda_build, cq, workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if local == 0:
+        cuda_build.build()
+    if world > 1:
+        dist.barrier()
+    cq.lib()
+
+    cfg = rank_config(rank)
+    X = wl.generate_activation(cfg)
+    T, I = X.shape
+    n = T * I
+    Xh = torch.from_numpy(X.view(np.int16)).view(torch.bfloat16)
+    Xd = Xh.cuda()
+    buf = cq.ActBuffers(T, I, torch.bfloat16, BITS)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+
+    def step():
+        cq.quantize_act(Xd, ALPHA, BITS, buffers=buf)
+
+    for _ in range(args.warmup):
+        flush.zero_()
+        step()
+    torch.cuda.synchronize()
+
+    K = args.steps
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    with ClockSampler(local, str(torch.cuda.get_device_properties(local).uuid)) as clocks:
+        for k in range(K):
+            flush.zero_()                         # untimed: evicts X and the outputs from L2
+            cq.set_timing_events(ev[k][2], ev[k][3])
+            ev[k][0].record()
+            step()
+            ev[k][1].record()
+        torch.cuda.synchronize()
+    cq.set_timing_events(None, None)
+    if world > 1:
+        dist.barrier()
+    step_ms = [e[0].elapsed_time(e[1]) for e in ev]
+    quant_ms = [e[2].elapsed_time(e[3]) for e in ev]
+    total_ms = torch.tensor([sum(step_ms)], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(total_ms, op=dist.ReduceOp.MAX)
+    total_ms = float(total_ms.item())
+    value = BYTES_PER_ELEMENT_STEP * n * K * world / (total_ms * 1e-3) / 1e9
+    zero_count = int(buf.zero_count.item())
+
+    # ---- end to end: host buffers in, host buffers out, through cq_quantize_act_host
+    Xp = Xh.pin_memory()
+    hb = cq.HostBuffers(T, I, torch.bfloat16, BITS)
+    Ke = max(1, args.e2e_steps)
+    for _ in range(2):
+        cq.quantize_act_host(Xp, ALPHA, BITS, buffers=hb)
+    torch.cuda.synchronize()
+    e0 = [torch.cuda.Event(enable_timing=True) for _ in range(Ke)]
+    e1 = [torch.cuda.Event(enable_timing=True) for _ in range(Ke)]
+    if world > 1:
+        dist.barrier()
+    for k in range(Ke):
+        e0[k].record()
+        cq.quantize_act_host(Xp, ALPHA, BITS, buffers=hb)
+        e1[k].record()
+    torch.cuda.synchronize()
+    e2e_ms = torch.tensor([sum(a.elapsed_time(b) for a, b in zip(e0, e1))], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
+    e2e_value = BYTES_PER_ELEMENT_STEP * n * Ke * world / (float(e2e_ms.item()) * 1e-3) / 1e9
+    assert int(hb.zero_count.item()) == zero_count
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peak()
+    quant_mean_ms = statistics.fmean(quant_ms)
+    achieved = BYTES_PER_ELEMENT_QUANT_PASS * n / (quant_mean_ms * 1e-3) / 1e9
+    traffic = NCU_TRAFFIC["bytes_per_launch"] if NCU_TRAFFIC["sources_sha256"] == kernel_sources_digest() else None
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
+        "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{cfg.name} {T}x{I} bf16 (LLaMA-70B MLP input), INT{BITS} codes + bf16 dequant + zero count, alpha={ALPHA}",
+                   "l2": "flushed between steps (256 MiB write, untimed); X (235 MB) also exceeds the 126 MB L2",
+                   "timing": "CUDA events per step on the launch stream, summed; max over ranks",
+                   "bytes_per_element": BYTES_PER_ELEMENT_STEP, "per_rank": "independent matrices, no collective"},
+        "elements_per_s": n * K * world / (total_ms * 1e-3),
+        "fraction_of_hbm_roofline": value / (peak * world),
+        "ms_per_step_median": statistics.median(step_ms),
+        "kernel_proportion": zero_count / n,
+        "clocks": clocks.summary(),
+        "gpu_launches": 3 * K,
+        "e2e": {"value": e2e_value, "unit": UNIT, "steps": Ke,
+                "h2d_bytes_per_step": X.nbytes, "d2h_bytes_per_step": hb.d2h_bytes(),
+                "api": "cq_quantize_act_host (pinned host buffers; copies inside the timed region)"},
+        "roofline": {"bound": "hbm", "kernel": "k3_quantize (quantize / pack / dequantize / zero-count pass)",
+                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": f"of {peak_kind}", "traffic": traffic,
+                     "algorithmic_bytes_per_launch": BYTES_PER_ELEMENT_QUANT_PASS * n,
+                     "avg_launch_ms": quant_mean_ms},
+    }
+
+    # ---- the oracle on the host cores, bounded sample of the same workload
+    from oracle import cq_oracle as orc
+    rows = 1024
+    Xs = X[:rows]
+    orc.quantize_act(X[:64], cfg.dtype, ALPHA, BITS, want_deq32=False)
+    t0 = time.perf_counter()
+    orc.quantize_act(Xs, cfg.dtype, ALPHA, BITS, want_deq32=False)
+    dt = time.perf_counter() - t0
+    out["cpu_baseline"] = {"value": BYTES_PER_ELEMENT_STEP * Xs.size / dt / 1e9, "unit": UNIT,
+                           "cores": orc.num_threads(), "kind": "oracle",
+                           "sample": f"first {rows} rows of the workload matrix ({rows}x{I}), one oracle quantize_act "
+                                     f"(t, c, codes, bf16 dequant, count), {dt:.2f} s"}
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

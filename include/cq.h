@@ -142,6 +142,11 @@ int cq_quantize_weight_per_channel(const void* W, int dtype, int64_t R, int64_t 
  * key: "k1_rows", "k3_rows".  value <= 0 restores the built-in choice.  Returns CQ_OK or CQ_ERR_SHAPE. */
 int cq_set_tuning(const char* key, int value);
 
+/* Measurement hook: while both are non-NULL, cq_quantize_act records the two cudaEvent_t (passed
+ * as void*, owned by the caller) on its stream immediately before and after the quantize pass, so
+ * that pass can be timed inside a real call.  Pass NULL, NULL to switch it off (the default). */
+int cq_set_timing_events(void* before_quantize_pass, void* after_quantize_pass);
+
 #ifdef __cplusplus
 }
 #endif

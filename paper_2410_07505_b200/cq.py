@@ -22,7 +22,7 @@ EXPORTS = (
     "cq_version", "cq_status_string", "cq_absmax_rows", "cq_absmax_cols", "cq_absmax_rows_cols",
     "cq_workspace_bytes", "cq_quantize_act", "cq_host_scratch_bytes", "cq_quantize_act_host",
     "cq_dequantize", "cq_kernel_count", "cq_kernel_count_x", "cq_quantize_weight_per_channel",
-    "cq_set_tuning",
+    "cq_set_tuning", "cq_set_timing_events",
 )
 
 
@@ -63,6 +63,7 @@ def lib() -> C.CDLL:
         L.cq_kernel_count_x.argtypes = [vp, ci, i64, i64, i64, dbl, ci, vp, vp, vp, vp, C.c_size_t, vp]
         L.cq_quantize_weight_per_channel.argtypes = [vp, ci, i64, i64, i64, ci, vp, vp, vp, ci, vp, vp]
         L.cq_set_tuning.argtypes = [C.c_char_p, ci]
+        L.cq_set_timing_events.argtypes = [vp, vp]
         for name in EXPORTS:
             if name not in ("cq_status_string", "cq_workspace_bytes", "cq_host_scratch_bytes"):
                 getattr(L, name).restype = ci
@@ -80,6 +81,14 @@ def status_string(status: int) -> str:
 
 def set_tuning(key: str, value: int) -> None:
     _check(lib().cq_set_tuning(key.encode(), int(value)), "cq_set_tuning")
+
+
+def set_timing_events(before: "torch.cuda.Event | None", after: "torch.cuda.Event | None") -> None:
+    """Have quantize_act record two (already created) CUDA events around its quantize pass."""
+    if before is None or after is None:
+        lib().cq_set_timing_events(None, None)
+    else:
+        lib().cq_set_timing_events(C.c_void_p(before.cuda_event), C.c_void_p(after.cuda_event))
 
 
 def _check(status: int, where: str) -> None:

@@ -299,6 +299,7 @@ g3_quantize(const uint16_t* __restrict__ X, int64_t T, int64_t I, int64_t ld, in
 // ============================================================================ host side
 static int g_tune_k1_rows = 0;
 static int g_tune_k3_rows = 0;
+static cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
 
 static inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
@@ -494,6 +495,8 @@ int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
     // ---- pass 2
     const bool any_out = codes != nullptr || deq != nullptr || zero_count != nullptr;
     if (any_out) {
+        const bool timed = g_ev_before != nullptr && g_ev_after != nullptr;
+        if (timed) cudaEventRecord(g_ev_before, st);
         if (fast_in && fast_out) {
             dim3 grid(p.nstrips, p.nrb3);
             const int deq_mode = deq == nullptr ? 0 : (deq_dtype == CQ_F32 ? 2 : 1);
@@ -516,6 +519,7 @@ int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
                 g3_quantize<CQ_BF16><<<blocks, kThreads, 0, st>>>(static_cast<const uint16_t*>(X), T, I, ld, bits, a_dev, b_dev,
                                                                   codes, deq, deq_dtype, zero_count);
         }
+        if (timed) cudaEventRecord(g_ev_after, st);
         if ((rc = launch_status()) != CQ_OK) return rc;
     }
     if (col_scale != nullptr && !b_in_place) {
@@ -555,6 +559,12 @@ int cq_set_tuning(const char* key, int value) {
     if (eq(key, k1)) { cq::g_tune_k1_rows = value > 0 ? value : 0; return CQ_OK; }
     if (eq(key, k3)) { cq::g_tune_k3_rows = value > 0 ? value : 0; return CQ_OK; }
     return CQ_ERR_SHAPE;
+}
+
+int cq_set_timing_events(void* before_quantize_pass, void* after_quantize_pass) {
+    cq::g_ev_before = static_cast<cudaEvent_t>(before_quantize_pass);
+    cq::g_ev_after = static_cast<cudaEvent_t>(after_quantize_pass);
+    return CQ_OK;
 }
 
 size_t cq_workspace_bytes(int64_t T, int64_t I) {
