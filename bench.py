@@ -203,6 +203,9 @@ def main() -> None:
 
     K = args.steps
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
+    for e in ev:                                   # torch creates the CUDA event on first record
+        e[2].record()
+        e[3].record()
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
