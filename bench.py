@@ -38,6 +38,7 @@ BYTES_PER_ELEMENT_STEP = 7.0        # X read twice (2+2) + int8 codes (1) + bf16
 BYTES_PER_ELEMENT_QUANT_PASS = 5.0  # quantize pass alone: X (2) + codes (1) + dequantized (2)
 FALLBACK_HBM_GBS = 6650.0
 L2_FLUSH_BYTES = 256 << 20
+HOOK_EVERY = 8
 
 # DRAM traffic of the quantize pass from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum
 # per launch), valid only for the kernel sources whose digest is recorded with it.
@@ -203,16 +204,22 @@ def main() -> None:
 
     K = args.steps
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
-    for e in ev:                                   # torch creates the CUDA event on first record
-        e[2].record()
-        e[3].record()
+    # The quantize pass is timed inside the real call on every HOOK_EVERY-th step only: the two extra
+    # event records sit between dependent kernels and cost a few microseconds of overlap.
+    hooked = [k for k in range(K) if k % HOOK_EVERY == 0]
+    for k in hooked:                               # torch creates the CUDA event on first record
+        ev[k][2].record()
+        ev[k][3].record()
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
     with ClockSampler(local, str(torch.cuda.get_device_properties(local).uuid)) as clocks:
         for k in range(K):
             flush.zero_()                         # untimed: evicts X and the outputs from L2
-            cq.set_timing_events(ev[k][2], ev[k][3])
+            if k % HOOK_EVERY == 0:
+                cq.set_timing_events(ev[k][2], ev[k][3])
+            elif k % HOOK_EVERY == 1:
+                cq.set_timing_events(None, None)
             ev[k][0].record()
             step()
             ev[k][1].record()
@@ -221,7 +228,7 @@ def main() -> None:
     if world > 1:
         dist.barrier()
     step_ms = [e[0].elapsed_time(e[1]) for e in ev]
-    quant_ms = [e[2].elapsed_time(e[3]) for e in ev]
+    quant_ms = [ev[k][2].elapsed_time(ev[k][3]) for k in hooked]
     total_ms = torch.tensor([sum(step_ms)], dtype=torch.float64, device="cuda")
     if world > 1:
         dist.all_reduce(total_ms, op=dist.ReduceOp.MAX)
@@ -282,7 +289,7 @@ def main() -> None:
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": f"of {peak_kind}", "traffic": traffic,
                      "algorithmic_bytes_per_launch": BYTES_PER_ELEMENT_QUANT_PASS * n,
-                     "avg_launch_ms": quant_mean_ms},
+                     "avg_launch_ms": quant_mean_ms, "launches_timed": len(hooked)},
     }
 
     # ---- the oracle on the host cores, bounded sample of the same workload

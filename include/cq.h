@@ -138,8 +138,10 @@ int cq_quantize_weight_per_channel(const void* W, int dtype, int64_t R, int64_t 
                                    void* codes, float* scale, void* deq, int deq_dtype,
                                    unsigned long long* zero_count, void* stream);
 
-/* Launch-shape knobs for measurement (rows per CTA of the two passes, CTAs per SM hints).
- * key: "k1_rows", "k3_rows".  value <= 0 restores the built-in choice.  Returns CQ_OK or CQ_ERR_SHAPE. */
+/* Launch-shape knobs for measurement.  key: "k1_ctas_per_sm", "k3_ctas_per_sm" (resident CTAs per SM
+ * the two passes size their grids for; 1..64), "k3_forward" (1: the quantize pass walks the rows in
+ * ascending order) or "no_pdl" (1: launch the quantize pass without programmatic dependent launch).  value <= 0 restores the built-in choice.  Results never depend on these.
+ * Returns CQ_OK or CQ_ERR_SHAPE. */
 int cq_set_tuning(const char* key, int value);
 
 /* Measurement hook: while both are non-NULL, cq_quantize_act records the two cudaEvent_t (passed

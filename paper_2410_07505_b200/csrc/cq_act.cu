@@ -1,11 +1,10 @@
 // CrossQuant activation quantizer: absmax pass, scale vectors, quantize pass (sm_100a).
 //
 // Pass 1 reads X once and produces partial row maxima (one per row and column strip) and partial
-// column maxima (one per column and row block) of the 15-bit magnitudes; the scale-vector kernel
-// finishes both reductions, so no atomics and no zero-initialisation are needed and the result does
-// not depend on scheduling.  Pass 2 re-reads X (from L2 where it still lives there: it walks the
-// row blocks in the opposite order), forms s_ij = a_i * b_j in registers and emits codes, the
-// dequantized matrix and the number of zero codes.
+// column maxima (one per column and resident CTA) of the 15-bit magnitudes; a small second kernel
+// finishes both reductions and writes t, c and the scale vectors, so no atomics or zero-initialised
+// buffers are involved and the result does not depend on scheduling.  Pass 2 re-reads X (walking the rows in the opposite order), forms
+// s_ij = a_i * b_j in registers and emits codes, the dequantized matrix and the number of zero codes.
 #include <math.h>
 
 #include <initializer_list>
@@ -13,46 +12,125 @@
 #include "cq_common.cuh"
 #include "cq_host.h"
 
+#ifndef CQ_K3_MIN_CTAS
+#define CQ_K3_MIN_CTAS 2
+#endif
+
 namespace cq {
 
+// ============================================================================ scale factors
+//   a_i = fl32(pow(t_i, alpha) / qmax), b_j = fl32(pow(c_j, 1 - alpha)) in fp64, with alpha in {0, 1}
+//   special-cased so that they reduce exactly to per-column / per-token quantization, plus the
+//   reciprocals the quantize pass uses for its candidate codes.
+__device__ __forceinline__ void row_scale_of(float ti, double alpha, int qmax, float& ai, float& rai) {
+    if (alpha == 1.0) ai = __fdiv_rn(ti, static_cast<float>(qmax));
+    else if (alpha == 0.0) ai = 1.0f;
+    else ai = static_cast<float>(pow(static_cast<double>(ti), alpha) / static_cast<double>(qmax));
+    rai = __fdiv_rn(1.0f, ai);
+}
+
+__device__ __forceinline__ void col_scale_of(float cj, double alpha, int qmax, float& bj, float& rbj) {
+    if (alpha == 1.0) bj = 1.0f;
+    else if (alpha == 0.0) bj = __fdiv_rn(cj, static_cast<float>(qmax));
+    else bj = static_cast<float>(pow(static_cast<double>(cj), 1.0 - alpha));
+    rbj = __fdiv_rn(1.0f, bj);
+}
+
 // ============================================================================ pass 1: absmax
-// Grid: x = column strip (blockDim.x vectors of 8 columns), y = row block of R rows.
-// ATOMIC = false: partial maxima to rowpart[T][nstrips] and colpart[nrb][I8*8] (16-bit magnitudes).
+// Grid: x = column strip (blockDim.x vectors of 8 columns), y = one of Y resident CTAs per strip.
+// CTA y walks the row groups (kG1 rows each) y, y+Y, y+2Y, ...  Each of its row slots is re-loaded
+// for the next group as soon as it has been consumed, so kG1 128-bit loads per thread stay in flight.  Threads past the last column re-read the last vector and rows past the end
+// re-read the last row: duplicates do not change a maximum.
+// ATOMIC = false: partial maxima to rowpart[T][nstrips] and colpart[Y][I8*8] (16-bit magnitudes).
 // ATOMIC = true : order-independent atomic max on the float bit patterns of t / c (pre-zeroed).
+#ifndef CQ_K1_GROUP_ROWS
+#define CQ_K1_GROUP_ROWS 4
+#endif
+constexpr int kG1 = CQ_K1_GROUP_ROWS; // rows per group of pass 1
+constexpr int kChunkGroups = 32;     // row maxima are flushed to global memory every 32 groups
+
 template <bool ATOMIC, int DT>
 __global__ void __launch_bounds__(kThreads)
-k1_absmax(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8, int R, int nstrips,
+k1_absmax(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8, int nstrips,
           uint16_t* __restrict__ rowpart, uint4* __restrict__ colpart,
           float* __restrict__ t, float* __restrict__ c) {
-    __shared__ uint16_t s_row[kThreads / 32][kMaxRowsPerCta];
+    __shared__ uint16_t s_row[kThreads / 32][kChunkGroups * kG1];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int v = blockIdx.x * blockDim.x + tid;
     const bool active = v < I8;
-    const int64_t r0 = static_cast<int64_t>(blockIdx.y) * R;
-    const int rows = static_cast<int>(min(static_cast<int64_t>(R), T - r0));
-    const uint4* p = X + r0 * ld8 + v;
+    const int64_t nfull = T / kG1;
+    const int64_t ngroups = (T + kG1 - 1) / kG1;
+    const int64_t Y = gridDim.y;
+    const uint4* xp = X + (active ? v : I8 - 1);
+    const int64_t step = kG1 * Y * ld8;
     uint4 cm = make_uint4(0, 0, 0, 0);
+    // The quantize pass may be scheduled onto SMs as this grid drains; it waits for this grid to
+    // complete (griddepcontrol.wait) before it touches anything written here.
+    asm volatile("griddepcontrol.launch_dependents;");
 
-    for (int r = 0; r < rows; r += 4) {
-        uint4 w[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            w[u] = make_uint4(0, 0, 0, 0);
-            if (active && r + u < rows) w[u] = ld_nc(p + u * ld8);
+    auto reduce_row = [&](const uint4& w, int slot) {
+        uint4 m = w;
+        m.x &= 0x7FFF7FFFu; m.y &= 0x7FFF7FFFu; m.z &= 0x7FFF7FFFu; m.w &= 0x7FFF7FFFu;
+        cm.x = max_u16x2(cm.x, m.x); cm.y = max_u16x2(cm.y, m.y);
+        cm.z = max_u16x2(cm.z, m.z); cm.w = max_u16x2(cm.w, m.w);
+        const uint32_t mm = max_u16x2(max_u16x2(m.x, m.y), max_u16x2(m.z, m.w));
+        const uint32_t wm = __reduce_max_sync(0xFFFFFFFFu, max(mm & 0xFFFFu, mm >> 16));
+        if (lane == 0) s_row[warp][slot] = static_cast<uint16_t>(wm);
+    };
+    auto flush_rows = [&](int64_t chunk_g0, int lg) {
+        __syncthreads();
+        const int nwarps = (blockDim.x + 31) >> 5;
+        for (int k = tid; k < lg * kG1; k += blockDim.x) {
+            const int64_t row = (chunk_g0 + static_cast<int64_t>(k / kG1) * Y) * kG1 + (k % kG1);
+            if (row < T) {
+                uint32_t m = 0;
+                for (int wdx = 0; wdx < nwarps; ++wdx) m = max(m, static_cast<uint32_t>(s_row[wdx][k]));
+                if constexpr (ATOMIC) {
+                    if (t != nullptr && m)
+                        atomicMax(reinterpret_cast<unsigned int*>(t) + row,
+                                  __float_as_uint(cvt16<DT>(static_cast<uint16_t>(m))));
+                } else {
+                    rowpart[row * nstrips + blockIdx.x] = static_cast<uint16_t>(m);
+                }
+            }
         }
-        p += 4 * ld8;
+        __syncthreads();
+    };
+
+    int64_t g = blockIdx.y;
+    int64_t chunk_g0 = g;
+    int lg = 0;
+    const uint4* p = xp + g * kG1 * ld8;
+    uint4 w[kG1];
+    if (g < nfull) {
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            uint4 m = w[u];
-            m.x &= 0x7FFF7FFFu; m.y &= 0x7FFF7FFFu; m.z &= 0x7FFF7FFFu; m.w &= 0x7FFF7FFFu;
-            cm.x = max_u16x2(cm.x, m.x); cm.y = max_u16x2(cm.y, m.y);
-            cm.z = max_u16x2(cm.z, m.z); cm.w = max_u16x2(cm.w, m.w);
-            uint32_t mm = max_u16x2(max_u16x2(m.x, m.y), max_u16x2(m.z, m.w));
-            uint32_t m16 = max(mm & 0xFFFFu, mm >> 16);
-            uint32_t wm = __reduce_max_sync(0xFFFFFFFFu, m16);
-            if (lane == 0 && r + u < rows) s_row[warp][r + u] = static_cast<uint16_t>(wm);
+        for (int u = 0; u < kG1; ++u) w[u] = ld_nc(p + u * ld8);
+    }
+    for (; g < ngroups; g += Y) {
+        if (g < nfull) {
+            const bool has_next = g + Y < nfull;
+            const uint4* pn = p + step;
+#pragma unroll
+            for (int u = 0; u < kG1; ++u) {
+                const uint4 cur = w[u];
+                if (has_next) w[u] = ld_nc(pn + u * ld8);
+                reduce_row(cur, lg * kG1 + u);
+            }
+            p = pn;
+        } else {                                   // the ragged last group: rows past T re-read row T-1
+#pragma unroll
+            for (int u = 0; u < kG1; ++u) {
+                const int64_t row = min(g * kG1 + u, T - 1);
+                reduce_row(ld_nc(xp + row * ld8), lg * kG1 + u);
+            }
+        }
+        if (++lg == kChunkGroups) {
+            flush_rows(chunk_g0, lg);
+            lg = 0;
+            chunk_g0 = g + Y;
         }
     }
+    if (lg > 0) flush_rows(chunk_g0, lg);
 
     if (active) {
         if constexpr (ATOMIC) {
@@ -62,25 +140,15 @@ k1_absmax(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8, int R, in
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     uint32_t lo = words[k] & 0xFFFFu, hi = words[k] >> 16;
-                    if (lo) atomicMax(cu + 2 * k, __float_as_uint(cvt16<DT>(static_cast<uint16_t>(lo))));
-                    if (hi) atomicMax(cu + 2 * k + 1, __float_as_uint(cvt16<DT>(static_cast<uint16_t>(hi))));
+                    // the plain read only skips atomics that could not raise the stored maximum
+                    const unsigned int flo = __float_as_uint(cvt16<DT>(static_cast<uint16_t>(lo)));
+                    const unsigned int fhi = __float_as_uint(cvt16<DT>(static_cast<uint16_t>(hi)));
+                    if (flo > __ldcg(cu + 2 * k)) atomicMax(cu + 2 * k, flo);
+                    if (fhi > __ldcg(cu + 2 * k + 1)) atomicMax(cu + 2 * k + 1, fhi);
                 }
             }
         } else {
             colpart[static_cast<int64_t>(blockIdx.y) * I8 + v] = cm;
-        }
-    }
-    __syncthreads();
-    const int nwarps = (blockDim.x + 31) >> 5;
-    for (int k = tid; k < rows; k += blockDim.x) {
-        uint32_t m = 0;
-        for (int wdx = 0; wdx < nwarps; ++wdx) m = max(m, static_cast<uint32_t>(s_row[wdx][k]));
-        if constexpr (ATOMIC) {
-            if (t != nullptr && m)
-                atomicMax(reinterpret_cast<unsigned int*>(t) + r0 + k,
-                          __float_as_uint(cvt16<DT>(static_cast<uint16_t>(m))));
-        } else {
-            rowpart[(r0 + k) * nstrips + blockIdx.x] = static_cast<uint16_t>(m);
         }
     }
 }
@@ -107,155 +175,266 @@ g1_absmax(const uint16_t* __restrict__ X, int64_t T, int64_t I, int64_t ld, int 
 }
 
 // ============================================================================ scale vectors
-// One thread per row (first T threads) or per column (next I threads).  Finishes the reductions of
-// pass 1 (from_partials) or takes t, c as given, then
-//   a_i = fl32(pow(t_i, alpha) / qmax), b_j = fl32(pow(c_j, 1 - alpha)) in fp64, with alpha in {0, 1}
-//   special-cased so that they reduce exactly to per-column / per-token quantization,
-// plus the reciprocals the quantize pass uses for its candidate codes.
+// From the partial maxima of pass 1.  CTAs [0, col_ctas): 256 columns each; thread (vx, grp) reduces
+// every 8th partial row of vector column vx, shared memory combines the 8 groups, then one thread per
+// column.  CTAs [col_ctas, ...): one thread per row.
 template <int DT>
 __global__ void __launch_bounds__(kThreads)
-k2_scales(int64_t T, int64_t I, int nstrips, int nrb, int64_t colpart_ld,
-          const uint16_t* __restrict__ rowpart, const uint16_t* __restrict__ colpart,
-          const float* __restrict__ t_in, const float* __restrict__ c_in,
-          double alpha, int qmax,
-          float* __restrict__ t_out, float* __restrict__ c_out,
-          float* __restrict__ a, float* __restrict__ b, float* __restrict__ ra, float* __restrict__ rb,
-          unsigned long long* __restrict__ zero_count) {
+k2_scales_from_partials(int64_t T, int64_t I, int I8, int nstrips, int Y, int col_ctas,
+                        const uint16_t* __restrict__ rowpart, const uint4* __restrict__ colpart,
+                        double alpha, int qmax,
+                        float* __restrict__ t_out, float* __restrict__ c_out,
+                        float* __restrict__ a, float* __restrict__ b, float* __restrict__ ra, float* __restrict__ rb,
+                        unsigned long long* __restrict__ zero_count) {
+    __shared__ uint4 s_part[8][32];
+    const int tid = threadIdx.x;
+    asm volatile("griddepcontrol.launch_dependents;");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (blockIdx.x == 0 && tid == 0 && zero_count != nullptr) *zero_count = 0ull;
+    if (static_cast<int>(blockIdx.x) < col_ctas) {
+        const int vx = tid & 31, grp = tid >> 5;
+        const int vcol = blockIdx.x * 32 + vx;
+        uint4 m = make_uint4(0, 0, 0, 0);
+        if (vcol < I8) {
+#pragma unroll 4
+            for (int y = grp; y < Y; y += 8) {
+                const uint4 w = colpart[static_cast<int64_t>(y) * I8 + vcol];
+                m.x = max_u16x2(m.x, w.x); m.y = max_u16x2(m.y, w.y);
+                m.z = max_u16x2(m.z, w.z); m.w = max_u16x2(m.w, w.w);
+            }
+        }
+        s_part[grp][vx] = m;
+        __syncthreads();
+        const int64_t j = static_cast<int64_t>(blockIdx.x) * 256 + tid;
+        if (j < I) {
+            const uint16_t* sp = reinterpret_cast<const uint16_t*>(&s_part[0][0]);
+            uint32_t mx = 0;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) mx = max(mx, static_cast<uint32_t>(sp[k * 256 + tid]));
+            const float cj = cvt16<DT>(static_cast<uint16_t>(mx));
+            if (c_out != nullptr) c_out[j] = cj;
+            float bj, rbj;
+            col_scale_of(cj, alpha, qmax, bj, rbj);
+            b[j] = bj;
+            rb[j] = rbj;
+        }
+    } else {
+        const int64_t i = static_cast<int64_t>(blockIdx.x - col_ctas) * kThreads + tid;
+        if (i < T) {
+            uint32_t m = 0;
+            for (int sx = 0; sx < nstrips; ++sx) m = max(m, static_cast<uint32_t>(rowpart[i * nstrips + sx]));
+            const float ti = cvt16<DT>(static_cast<uint16_t>(m));
+            if (t_out != nullptr) t_out[i] = ti;
+            float ai, rai;
+            row_scale_of(ti, alpha, qmax, ai, rai);
+            a[i] = ai;
+            ra[i] = rai;
+        }
+    }
+}
+
+// From finished t, c (the general path, and callers that supply the absmax vectors): one thread
+// per row (first T threads) or per column (next I threads).
+__global__ void __launch_bounds__(kThreads)
+k2_scales_from_vectors(int64_t T, int64_t I, const float* __restrict__ t_in, const float* __restrict__ c_in,
+                       double alpha, int qmax,
+                       float* __restrict__ a, float* __restrict__ b, float* __restrict__ ra, float* __restrict__ rb,
+                       unsigned long long* __restrict__ zero_count) {
     const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (idx == 0 && zero_count != nullptr) *zero_count = 0ull;
-    const float qmaxf = static_cast<float>(qmax);
     if (idx < T) {
-        float ti;
-        if (rowpart != nullptr) {
-            uint32_t m = 0;
-            for (int s = 0; s < nstrips; ++s) m = max(m, static_cast<uint32_t>(rowpart[idx * nstrips + s]));
-            ti = cvt16<DT>(static_cast<uint16_t>(m));
-        } else {
-            ti = t_in[idx];
-        }
-        if (t_out != nullptr) t_out[idx] = ti;
-        float ai;
-        if (alpha == 1.0) ai = __fdiv_rn(ti, qmaxf);
-        else if (alpha == 0.0) ai = 1.0f;
-        else ai = static_cast<float>(pow(static_cast<double>(ti), alpha) / static_cast<double>(qmax));
+        float ai, rai;
+        row_scale_of(t_in[idx], alpha, qmax, ai, rai);
         a[idx] = ai;
-        ra[idx] = __fdiv_rn(1.0f, ai);
+        ra[idx] = rai;
     } else if (idx - T < I) {
         const int64_t j = idx - T;
-        float cj;
-        if (colpart != nullptr) {
-            uint32_t m = 0;
-            for (int rbk = 0; rbk < nrb; ++rbk) m = max(m, static_cast<uint32_t>(colpart[rbk * colpart_ld + j]));
-            cj = cvt16<DT>(static_cast<uint16_t>(m));
-        } else {
-            cj = c_in[j];
-        }
-        if (c_out != nullptr) c_out[j] = cj;
-        float bj;
-        if (alpha == 1.0) bj = 1.0f;
-        else if (alpha == 0.0) bj = __fdiv_rn(cj, qmaxf);
-        else bj = static_cast<float>(pow(static_cast<double>(cj), 1.0 - alpha));
+        float bj, rbj;
+        col_scale_of(c_in[j], alpha, qmax, bj, rbj);
         b[j] = bj;
-        rb[j] = __fdiv_rn(1.0f, bj);
+        rb[j] = rbj;
     }
 }
 
 // ============================================================================ pass 2: quantize
-// Same tiling as pass 1; row blocks are visited in descending order.  Per thread and row: one
-// 128-bit load of 8 elements, s = a_i b_j, candidate code through the reciprocal product, exact
-// IEEE division only for the rare elements the residual test cannot decide.
+// Outside [2^-60, 2^60] a scale factor or its reciprocal may have lost relative precision (fp32
+// subnormals); such rows and columns are never trusted to the candidate test.
+constexpr float kScaleLo = 8.6736173798840355e-19f;    // 2^-60
+constexpr float kScaleHi = 1.152921504606846976e18f;   // 2^60
+// The candidate q = round-half-even(v), v = x * (1/a_i) * (1/b_j), is accepted when |v - q| < 1/2 - 2^-12.
+// With a_i, b_j, their reciprocals and s_ij all normal, v differs from z = x / s_ij by less than
+// 5 * 2^-24 |z| <= 2^-14.6 (|z| <= 128), so |z - q| < 1/2 - 2^-12 + 2^-14.6 and the IEEE quotient
+// fl32(z), which lies within 2^-17 of z, rounds to the same q; |z| <= qmax (1 + 2^-22) keeps q in range.
+constexpr float kAcceptBelow = 0.499755859375f;         // 1/2 - 2^-12
+
+// Eight elements of one row in packed fp32x2 arithmetic (bit-identical to the scalar IEEE operations,
+// half the issue slots).  y2[k] = kMagic + q and q2[k] = q for elements 2k, 2k+1.
+template <int DT, int BITS>
+__device__ __forceinline__ void quantize_row8(const uint4& w, float a, float ra, const float2 (&b2)[4],
+                                              const float2 (&rb2)[4], bool row_safe,
+                                              float2 (&y2)[4], float2 (&q2)[4]) {
+    constexpr float qmaxf = static_cast<float>((1 << (BITS - 1)) - 1);
+    const float2 ra2 = make_float2(ra, ra);
+    const float2 m2 = make_float2(kMagic, kMagic), nm2 = make_float2(-kMagic, -kMagic);
+    const float2 neg1 = make_float2(-1.0f, -1.0f);
+    const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+    float worst = 0.0f;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const float2 x = unpack16x2<DT>(words[k]);
+        const float2 r = __fmul2_rn(ra2, rb2[k]);
+        const float2 v = __fmul2_rn(x, r);                    // x / s, approximately
+        y2[k] = __fadd2_rn(v, m2);
+        q2[k] = __fadd2_rn(y2[k], nm2);                       // round-half-even(v), exact
+        const float2 f = __ffma2_rn(q2[k], neg1, v);          // v - q, exact
+        worst = fmaxf(fmaxf(worst, fabsf(f.x)), fabsf(f.y));
+    }
+    if (!(row_safe && worst < kAcceptBelow)) {
+        // Rare: some element is too close to a rounding boundary (or a scale is extreme / zero / NaN)
+        // for the cheap test to decide.  Re-examine each element with the exact residual; the
+        // undecided ones take the defining sequence (IEEE division, round half to even, clamp).
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float2 x = unpack16x2<DT>(words[k]);
+            const float xs[2] = {x.x, x.y};
+            const float bs[2] = {b2[k].x, b2[k].y};
+            const float rs[2] = {rb2[k].x, rb2[k].y};
+            float ys[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const float sh = __fmul_rn(a, bs[h]);
+                bool good;
+                ys[h] = quant_candidate(xs[h], sh, __fmul_rn(ra, rs[h]), qmaxf, good);
+                good = good && a >= kScaleLo && bs[h] >= kScaleLo && sh >= kScaleLo;
+                if (!good) ys[h] = quant_exact(xs[h], sh, qmaxf);
+            }
+            y2[k] = make_float2(ys[0], ys[1]);
+            q2[k] = __fadd2_rn(y2[k], nm2);
+        }
+    }
+}
+
+// Same strip / resident-CTA layout and rolling four-row prefetch as pass 1.  Full row groups are
+// walked from the last one backwards (the rows pass 1 touched last are the likeliest to be still in
+// L2) unless `forward` is set; a ragged last group (T not a multiple of 4) is done first by CTA y = 0.
+// Lanes past the last column compute on the last vector and store nothing.
 // DEQ: 0 none, 1 same 16-bit type as X, 2 fp32.
 template <int DT, int BITS, int DEQ, bool CODES, bool COUNT>
-__global__ void __launch_bounds__(kThreads, 3)
-k3_quantize(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8, int R,
+__global__ void __launch_bounds__(kThreads, CQ_K3_MIN_CTAS)
+k3_quantize(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
             const float* __restrict__ a, const float* __restrict__ ra,
             const float* __restrict__ b, const float* __restrict__ rb,
             void* __restrict__ codes, void* __restrict__ deq,
-            unsigned long long* __restrict__ zero_count) {
-    constexpr float qmaxf = static_cast<float>((1 << (BITS - 1)) - 1);
-    const int tid = threadIdx.x;
+            unsigned long long* __restrict__ zero_count, int forward) {
+    const int tid = threadIdx.x, lane = tid & 31;
     const int v = blockIdx.x * blockDim.x + tid;
     const bool active = v < I8;
-    const int64_t rblk = static_cast<int64_t>(gridDim.y - 1 - blockIdx.y);
-    const int64_t r0 = rblk * R;
-    const int rows = static_cast<int>(min(static_cast<int64_t>(R), T - r0));
+    const bool warp_active = (v - lane) < I8;
+    const int vv = active ? v : I8 - 1;
+    const int64_t nfull = T >> 2;
+    const int64_t Y = gridDim.y;
     unsigned int zeros = 0;
 
-    if (active) {
-        float bj[8], rbj[8];
+    // Everything this kernel reads except X is produced by the preceding kernel of the stream.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
+    if (warp_active) {
+        float2 b2[4], rb2[4];
+        float bmin;
         {
-            const float4* bp = reinterpret_cast<const float4*>(b) + static_cast<int64_t>(v) * 2;
-            const float4* rp = reinterpret_cast<const float4*>(rb) + static_cast<int64_t>(v) * 2;
-            float4 b0 = __ldg(bp), b1 = __ldg(bp + 1), q0 = __ldg(rp), q1 = __ldg(rp + 1);
-            bj[0] = b0.x; bj[1] = b0.y; bj[2] = b0.z; bj[3] = b0.w;
-            bj[4] = b1.x; bj[5] = b1.y; bj[6] = b1.z; bj[7] = b1.w;
-            rbj[0] = q0.x; rbj[1] = q0.y; rbj[2] = q0.z; rbj[3] = q0.w;
-            rbj[4] = q1.x; rbj[5] = q1.y; rbj[6] = q1.z; rbj[7] = q1.w;
+            const float4* bp = reinterpret_cast<const float4*>(b) + static_cast<int64_t>(vv) * 2;
+            const float4* rp = reinterpret_cast<const float4*>(rb) + static_cast<int64_t>(vv) * 2;
+            const float4 b0 = __ldg(bp), b1 = __ldg(bp + 1), q0 = __ldg(rp), q1 = __ldg(rp + 1);
+            b2[0] = make_float2(b0.x, b0.y); b2[1] = make_float2(b0.z, b0.w);
+            b2[2] = make_float2(b1.x, b1.y); b2[3] = make_float2(b1.z, b1.w);
+            rb2[0] = make_float2(q0.x, q0.y); rb2[1] = make_float2(q0.z, q0.w);
+            rb2[2] = make_float2(q1.x, q1.y); rb2[3] = make_float2(q1.z, q1.w);
+            bmin = fminf(fminf(fminf(b0.x, b0.y), fminf(b0.z, b0.w)), fminf(fminf(b1.x, b1.y), fminf(b1.z, b1.w)));
+            const float bmax = fmaxf(fmaxf(fmaxf(b0.x, b0.y), fmaxf(b0.z, b0.w)), fmaxf(fmaxf(b1.x, b1.y), fmaxf(b1.z, b1.w)));
+            if (!(bmin >= kScaleLo && bmax <= kScaleHi)) bmin = 0.0f;      // never trust this thread's columns
         }
-        const uint4* p = X + r0 * ld8 + v;
-        for (int r = 0; r < rows; r += 4) {
-            uint4 w[4];
-            float ar[4], rar[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                if (r + u < rows) {
-                    w[u] = ld_stream(p + u * ld8);
-                    ar[u] = __ldg(a + r0 + r + u);
-                    rar[u] = __ldg(ra + r0 + r + u);
-                }
+        const uint4* xp = X + vv;
+
+        // one row of 8 elements: quantize, pack, store (stores only from lanes that own a column)
+        auto do_row = [&](const uint4& wrow, float au, float rau, int64_t vec) {
+            const bool row_safe = au >= kScaleLo && au <= kScaleHi && __fmul_rn(au, bmin) >= kScaleLo;
+            float2 y2[4], q2[4];
+            quantize_row8<DT, BITS>(wrow, au, rau, b2, rb2, row_safe, y2, q2);
+            if constexpr (BITS == 8) {
+                const uint32_t c0 = pack_int8x4(y2[0].x, y2[0].y, y2[1].x, y2[1].y);
+                const uint32_t c1 = pack_int8x4(y2[2].x, y2[2].y, y2[3].x, y2[3].y);
+                if constexpr (COUNT) zeros += zero_bytes(c0) + zero_bytes(c1);
+                if constexpr (CODES) { if (active) st_stream(reinterpret_cast<uint2*>(codes) + vec, make_uint2(c0, c1)); }
+            } else {
+                const float ys[8] = {y2[0].x, y2[0].y, y2[1].x, y2[1].y, y2[2].x, y2[2].y, y2[3].x, y2[3].y};
+                const uint32_t c0 = pack_int4x8(ys);
+                if constexpr (COUNT) zeros += zero_nibbles(c0);
+                if constexpr (CODES) { if (active) st_stream(reinterpret_cast<uint32_t*>(codes) + vec, c0); }
             }
-            p += 4 * ld8;
+            if constexpr (DEQ != 0) {
+                const float2 a2 = make_float2(au, au);
+                float2 d2[4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                if (r + u >= rows) break;
-                const int64_t row = r0 + r + u;
-                const uint32_t words[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
-                float x[8], y[8];
-                unsigned int bad = 0;
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    float2 f = unpack16x2<DT>(words[k]);
-                    x[2 * k] = f.x; x[2 * k + 1] = f.y;
-                }
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    bool ok;
-                    y[e] = quant_candidate(x[e], __fmul_rn(ar[u], bj[e]), __fmul_rn(rar[u], rbj[e]), qmaxf, ok);
-                    bad |= (ok ? 0u : 1u) << e;
-                }
-                if (bad) {
-#pragma unroll
-                    for (int e = 0; e < 8; ++e)
-                        if ((bad >> e) & 1u) y[e] = quant_exact(x[e], __fmul_rn(ar[u], bj[e]), qmaxf);
-                }
-                const int64_t vec = row * I8 + v;
-                if constexpr (BITS == 8) {
-                    uint32_t c0 = pack_int8x4(y[0], y[1], y[2], y[3]);
-                    uint32_t c1 = pack_int8x4(y[4], y[5], y[6], y[7]);
-                    if constexpr (COUNT) zeros += zero_bytes(c0) + zero_bytes(c1);
-                    if constexpr (CODES) st_stream(reinterpret_cast<uint2*>(codes) + vec, make_uint2(c0, c1));
+                for (int k = 0; k < 4; ++k) d2[k] = __fmul2_rn(q2[k], __fmul2_rn(a2, b2[k]));
+                if constexpr (DEQ == 1) {
+                    uint4 o;
+                    o.x = pack16x2<DT>(d2[0].x, d2[0].y); o.y = pack16x2<DT>(d2[1].x, d2[1].y);
+                    o.z = pack16x2<DT>(d2[2].x, d2[2].y); o.w = pack16x2<DT>(d2[3].x, d2[3].y);
+                    if (active) st_stream(reinterpret_cast<uint4*>(deq) + vec, o);
                 } else {
-                    uint32_t c0 = pack_int4x8(y);
-                    if constexpr (COUNT) zeros += zero_nibbles(c0);
-                    if constexpr (CODES) st_stream(reinterpret_cast<uint32_t*>(codes) + vec, c0);
-                }
-                if constexpr (DEQ != 0) {
-                    float d[8];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) d[e] = __fmul_rn(code_as_float(y[e]), __fmul_rn(ar[u], bj[e]));
-                    if constexpr (DEQ == 1) {
-                        uint4 o;
-                        o.x = pack16x2<DT>(d[0], d[1]); o.y = pack16x2<DT>(d[2], d[3]);
-                        o.z = pack16x2<DT>(d[4], d[5]); o.w = pack16x2<DT>(d[6], d[7]);
-                        st_stream(reinterpret_cast<uint4*>(deq) + vec, o);
-                    } else {
-                        float4* o = reinterpret_cast<float4*>(deq) + vec * 2;
-                        st_stream(o, make_float4(d[0], d[1], d[2], d[3]));
-                        st_stream(o + 1, make_float4(d[4], d[5], d[6], d[7]));
+                    float4* o = reinterpret_cast<float4*>(deq) + vec * 2;
+                    if (active) {
+                        st_stream(o, make_float4(d2[0].x, d2[0].y, d2[1].x, d2[1].y));
+                        st_stream(o + 1, make_float4(d2[2].x, d2[2].y, d2[3].x, d2[3].y));
                     }
                 }
             }
+        };
+        // lanes 0-3 fetch a_i of a group's four rows, lanes 4-7 the reciprocals (rows clamped to T-1)
+        auto load_scales = [&](int64_t g) {
+            const int64_t row = min((g << 2) + (lane & 3), T - 1);
+            return lane < 8 ? __ldg((lane < 4 ? a : ra) + row) : 0.0f;
+        };
+
+        if ((T & 3) != 0 && blockIdx.y == 0) {          // ragged last group
+            const float arv = load_scales(nfull);
+            for (int u = 0; u < static_cast<int>(T & 3); ++u) {
+                const int64_t row = (nfull << 2) + u;
+                const uint4 wrow = ld_stream(xp + row * ld8);
+                do_row(wrow, __shfl_sync(0xFFFFFFFFu, arv, u), __shfl_sync(0xFFFFFFFFu, arv, 4 + u), row * I8 + vv);
+            }
         }
+
+        int64_t pos = blockIdx.y;
+        if (pos < nfull) {
+            const int64_t dgroups = forward ? Y : -Y;
+            int64_t g = forward ? pos : nfull - 1 - pos;
+            const int64_t xstep = 4 * dgroups * ld8, ostep = 4 * dgroups * static_cast<int64_t>(I8);
+            const uint4* p = xp + (g << 2) * ld8;
+            int64_t vec = (g << 2) * I8 + vv;
+            uint4 w[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) w[u] = ld_stream(p + u * ld8);
+            float arv = load_scales(g);
+            for (; pos < nfull; pos += Y) {
+                const bool has_next = pos + Y < nfull;
+                const uint4* pn = p + xstep;
+                float arvn = 0.0f;
+                if (has_next) arvn = load_scales(g + dgroups);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const uint4 cur = w[u];
+                    if (has_next) w[u] = ld_stream(pn + u * ld8);
+                    do_row(cur, __shfl_sync(0xFFFFFFFFu, arv, u), __shfl_sync(0xFFFFFFFFu, arv, 4 + u),
+                           vec + static_cast<int64_t>(u) * I8);
+                }
+                p = pn;
+                vec += ostep;
+                g += dgroups;
+                arv = arvn;
+            }
+        }
+        if (!active) zeros = 0;
     }
     if constexpr (COUNT) cta_count_add(zeros, zero_count);
 }
@@ -297,11 +476,22 @@ g3_quantize(const uint16_t* __restrict__ X, int64_t T, int64_t I, int64_t ld, in
 }
 
 // ============================================================================ host side
-static int g_tune_k1_rows = 0;
-static int g_tune_k3_rows = 0;
+static int g_tune_k1_ctas = 0;      // resident CTAs per SM assumed for pass 1 (0 = ask the runtime)
+static int g_tune_k3_ctas = 0;      // the same for pass 2
+static int g_tune_k3_forward = 0;   // walk pass 2 in ascending row order
+static int g_tune_no_pdl = 0;       // launch pass 2 without programmatic dependent launch
 static cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
 
 static inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
+
+// Upper bound on the CTAs per column strip of pass 1 (= rows of the column-partial buffer): keeps
+// that buffer at 8 MiB or less whatever the device.
+static int y_cap(int I8) {
+    int64_t cap = (int64_t(8) << 20) / (static_cast<int64_t>(I8 > 0 ? I8 : 1) * 16);
+    if (cap < 8) cap = 8;
+    if (cap > 2048) cap = 2048;
+    return static_cast<int>(cap);
+}
 
 Plan make_plan(int64_t T, int64_t I) {
     Plan p{};
@@ -316,16 +506,8 @@ Plan make_plan(int64_t T, int64_t I) {
         }
     }
     p.nstrips = p.I8 > 0 ? (p.I8 + p.W - 1) / p.W : 1;
-    // pass 1: about one resident wave (8 CTAs of 256 threads per SM, 148 SMs)
-    int r1 = g_tune_k1_rows > 0 ? g_tune_k1_rows
-                                : static_cast<int>((T * p.nstrips + 1183) / 1184);
-    r1 = round_up(r1 < 16 ? 16 : r1, 4);
-    p.R1 = r1 > kMaxRowsPerCta ? kMaxRowsPerCta : r1;
-    p.nrb1 = static_cast<int>(T > 0 ? (T + p.R1 - 1) / p.R1 : 1);
-    int r3 = g_tune_k3_rows > 0 ? g_tune_k3_rows : 16;
-    r3 = round_up(r3, 4);
-    p.R3 = r3 > 4096 ? 4096 : r3;
-    p.nrb3 = static_cast<int>(T > 0 ? (T + p.R3 - 1) / p.R3 : 1);
+    p.ngroups = (T + 3) / 4;
+    p.ycap = y_cap(p.I8);
 
     auto carve = [&](size_t bytes) { size_t off = p.total; p.total += (bytes + 255) / 256 * 256; return off; };
     p.total = 0;
@@ -335,10 +517,10 @@ Plan make_plan(int64_t T, int64_t I) {
     p.off_b = carve(sizeof(float) * static_cast<size_t>(p.I8) * 8);
     p.off_ra = carve(sizeof(float) * static_cast<size_t>(T));
     p.off_rb = carve(sizeof(float) * static_cast<size_t>(p.I8) * 8);
-    // sized for the finest pass-1 tiling the tuning knob can select (16 rows per CTA)
-    size_t max_nrb = static_cast<size_t>((T + 15) / 16 + 1);
+    p.off_counters = carve(sizeof(unsigned int) * (static_cast<size_t>(p.nstrips) + 65536));
     p.off_rowpart = carve(sizeof(uint16_t) * static_cast<size_t>(T) * p.nstrips);
-    p.off_colpart = carve(sizeof(uint16_t) * max_nrb * static_cast<size_t>(p.I8) * 8);
+    const int64_t ymax = p.ngroups < p.ycap ? (p.ngroups > 0 ? p.ngroups : 1) : p.ycap;
+    p.off_colpart = carve(sizeof(uint16_t) * static_cast<size_t>(ymax) * static_cast<size_t>(p.I8) * 8);
     return p;
 }
 
@@ -346,7 +528,7 @@ static bool aligned(const void* p, size_t n) { return (reinterpret_cast<uintptr_
 
 int check_matrix(const void* X, int dtype, int64_t T, int64_t I, int64_t ld) {
     if (T < 0 || I < 0 || ld < I) return CQ_ERR_SHAPE;
-    if (T > (int64_t(1) << 31) - 1 - kMaxRowsPerCta || I > (int64_t(1) << 31) - 64) return CQ_ERR_SHAPE;
+    if (T > (int64_t(1) << 31) - 1024 || I > (int64_t(1) << 31) - 64) return CQ_ERR_SHAPE;
     if (dtype != CQ_F16 && dtype != CQ_BF16) return CQ_ERR_DTYPE;
     if (T > 0 && I > 0) {
         if (X == nullptr) return CQ_ERR_NULL;
@@ -361,6 +543,37 @@ static bool fast_input(const void* X, int64_t I, int64_t ld) {
 
 static int launch_status() { return cudaGetLastError() == cudaSuccess ? CQ_OK : CQ_ERR_CUDA; }
 
+static int sm_count() {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+        n = 148;
+    return n;
+}
+
+// CTAs per column strip so that the whole grid is resident at once: floor(SMs * CTAs/SM / strips).
+template <typename Kernel>
+static int resident_y(Kernel kern, int W, int nstrips, int64_t ngroups, int tuned_ctas_per_sm, int cap) {
+    int per_sm = tuned_ctas_per_sm;
+    if (per_sm <= 0 && cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, W, 0) != cudaSuccess) per_sm = 1;
+    if (per_sm < 1) per_sm = 1;
+    int64_t y = static_cast<int64_t>(sm_count()) * per_sm / nstrips;
+    if (y > ngroups) y = ngroups;
+    if (cap > 0 && y > cap) y = cap;
+    if (y > 65535) y = 65535;
+    if (y < 1) y = 1;
+    return static_cast<int>(y);
+}
+
+template <bool ATOMIC, int DT>
+static int launch_k1(const Plan& p, const void* X, int64_t T, int64_t ld, uint16_t* rowpart, uint16_t* colpart,
+                     float* t, float* c, cudaStream_t st) {
+    auto kern = k1_absmax<ATOMIC, DT>;
+    const int Y = resident_y(kern, p.W, p.nstrips, (p.ngroups * 4 + kG1 - 1) / kG1, g_tune_k1_ctas, ATOMIC ? 0 : p.ycap);
+    kern<<<dim3(p.nstrips, Y), p.W, 0, st>>>(static_cast<const uint4*>(X), T, p.I8, ld / 8, p.nstrips, rowpart,
+                                             reinterpret_cast<uint4*>(colpart), t, c);
+    return Y;
+}
+
 // pass 1 with atomics into pre-zeroed t / c (either may be null)
 static int absmax_atomic(const void* X, int dtype, int64_t T, int64_t I, int64_t ld, float* t, float* c,
                          cudaStream_t st) {
@@ -369,13 +582,8 @@ static int absmax_atomic(const void* X, int dtype, int64_t T, int64_t I, int64_t
     if (T == 0 || I == 0) return CQ_OK;
     Plan p = make_plan(T, I);
     if (fast_input(X, I, ld)) {
-        dim3 grid(p.nstrips, p.nrb1);
-        if (dtype == CQ_F16)
-            k1_absmax<true, CQ_F16><<<grid, p.W, 0, st>>>(static_cast<const uint4*>(X), T, p.I8, ld / 8, p.R1,
-                                                            p.nstrips, nullptr, nullptr, t, c);
-        else
-            k1_absmax<true, CQ_BF16><<<grid, p.W, 0, st>>>(static_cast<const uint4*>(X), T, p.I8, ld / 8, p.R1,
-                                                             p.nstrips, nullptr, nullptr, t, c);
+        if (dtype == CQ_F16) launch_k1<true, CQ_F16>(p, X, T, ld, nullptr, nullptr, t, c, st);
+        else launch_k1<true, CQ_BF16>(p, X, T, ld, nullptr, nullptr, t, c, st);
     } else {
         const int R = 64;
         dim3 grid(static_cast<unsigned>((I + kThreads - 1) / kThreads), static_cast<unsigned>((T + R - 1) / R));
@@ -387,26 +595,51 @@ static int absmax_atomic(const void* X, int dtype, int64_t T, int64_t I, int64_t
     return launch_status();
 }
 
+// Programmatic dependent launch: the kernel's CTAs may become resident while the previous kernel of
+// the stream drains; the kernel itself waits (griddepcontrol.wait) before reading what that one wrote.
+template <typename... KArgs, typename... Args>
+static void launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = g_tune_no_pdl ? 0 : 1;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
+struct K3Args {
+    const uint4* X; int64_t T; int I8; int64_t ld8;
+    const float *a, *ra, *b, *rb;
+    void* codes; void* deq; unsigned long long* zc;
+};
+
+template <int DT, int BITS, int DEQ, bool CODES, bool COUNT>
+static void launch_k3_one(const Plan& p, const K3Args& k, cudaStream_t st) {
+    auto kern = k3_quantize<DT, BITS, DEQ, CODES, COUNT>;
+    const int Y = resident_y(kern, p.W, p.nstrips, p.ngroups, g_tune_k3_ctas, 0);
+    launch_dependent(kern, dim3(p.nstrips, Y), dim3(p.W), st, k.X, k.T, k.I8, k.ld8, k.a, k.ra, k.b, k.rb, k.codes,
+                     k.deq, k.zc, g_tune_k3_forward);
+}
+
 template <int DT, int BITS, int DEQ>
-static void launch_k3(bool has_codes, bool has_count, dim3 grid, int W, cudaStream_t st, const uint4* X, int64_t T,
-                      int I8, int64_t ld8, int R, const float* a, const float* ra, const float* b, const float* rb,
-                      void* codes, void* deq, unsigned long long* zc) {
-    if (has_codes) {
-        if (has_count) k3_quantize<DT, BITS, DEQ, true, true><<<grid, W, 0, st>>>(X, T, I8, ld8, R, a, ra, b, rb, codes, deq, zc);
-        else k3_quantize<DT, BITS, DEQ, true, false><<<grid, W, 0, st>>>(X, T, I8, ld8, R, a, ra, b, rb, codes, deq, zc);
-    } else {
-        if (has_count) k3_quantize<DT, BITS, DEQ, false, true><<<grid, W, 0, st>>>(X, T, I8, ld8, R, a, ra, b, rb, codes, deq, zc);
-        else k3_quantize<DT, BITS, DEQ, false, false><<<grid, W, 0, st>>>(X, T, I8, ld8, R, a, ra, b, rb, codes, deq, zc);
-    }
+static void launch_k3_flags(const Plan& p, const K3Args& k, cudaStream_t st) {
+    const bool hc = k.codes != nullptr, hz = k.zc != nullptr;
+    if (hc && hz) launch_k3_one<DT, BITS, DEQ, true, true>(p, k, st);
+    else if (hc) launch_k3_one<DT, BITS, DEQ, true, false>(p, k, st);
+    else if (hz) launch_k3_one<DT, BITS, DEQ, false, true>(p, k, st);
+    else launch_k3_one<DT, BITS, DEQ, false, false>(p, k, st);
 }
 
 template <int DT, int BITS>
-static void launch_k3_deq(int deq_mode, bool has_codes, bool has_count, dim3 grid, int W, cudaStream_t st,
-                          const uint4* X, int64_t T, int I8, int64_t ld8, int R, const float* a, const float* ra,
-                          const float* b, const float* rb, void* codes, void* deq, unsigned long long* zc) {
-    if (deq_mode == 0) launch_k3<DT, BITS, 0>(has_codes, has_count, grid, W, st, X, T, I8, ld8, R, a, ra, b, rb, codes, deq, zc);
-    else if (deq_mode == 1) launch_k3<DT, BITS, 1>(has_codes, has_count, grid, W, st, X, T, I8, ld8, R, a, ra, b, rb, codes, deq, zc);
-    else launch_k3<DT, BITS, 2>(has_codes, has_count, grid, W, st, X, T, I8, ld8, R, a, ra, b, rb, codes, deq, zc);
+static void launch_k3_deq(const Plan& p, const K3Args& k, int deq_mode, cudaStream_t st) {
+    if (deq_mode == 0) launch_k3_flags<DT, BITS, 0>(p, k, st);
+    else if (deq_mode == 1) launch_k3_flags<DT, BITS, 1>(p, k, st);
+    else launch_k3_flags<DT, BITS, 2>(p, k, st);
 }
 
 // Shared body of cq_quantize_act and cq_kernel_count_x.  t_given/c_given: skip pass 1.
@@ -440,7 +673,8 @@ int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
     // as whole float4 pairs, so col_scale must be 16-byte aligned to be used in place.
     const bool given = t_given != nullptr && c_given != nullptr;
     float* t_dev = t != nullptr ? t : reinterpret_cast<float*>(ws + p.off_t);
-    float* c_dev = c != nullptr ? c : reinterpret_cast<float*>(ws + p.off_c);
+    const bool c_in_place = c != nullptr;
+    float* c_dev = c_in_place ? c : reinterpret_cast<float*>(ws + p.off_c);
     float* a_dev = row_scale != nullptr ? row_scale : reinterpret_cast<float*>(ws + p.off_a);
     const bool b_in_place = col_scale != nullptr && aligned(col_scale, 16);
     float* b_dev = b_in_place ? col_scale : reinterpret_cast<float*>(ws + p.off_b);
@@ -453,42 +687,32 @@ int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
     const bool fast_in = fast_input(X, I, ld);
     const bool fast_out = (codes == nullptr || aligned(codes, bits == 8 ? 8 : 4)) &&
                           (deq == nullptr || aligned(deq, 16));
-    const int64_t n2 = T + I;
-    const unsigned k2_blocks = static_cast<unsigned>((n2 + kThreads - 1) / kThreads);
+    const unsigned k2v_blocks = static_cast<unsigned>((T + I + kThreads - 1) / kThreads);
 
     // ---- pass 1 + scale vectors
     if (given) {
-        if (dtype == CQ_F16)
-            k2_scales<CQ_F16><<<k2_blocks, kThreads, 0, st>>>(T, I, 0, 0, 0, nullptr, nullptr, t_given, c_given, alpha,
-                                                              qmax, t, c, a_dev, b_dev, ra_dev, rb_dev, zero_count);
-        else
-            k2_scales<CQ_BF16><<<k2_blocks, kThreads, 0, st>>>(T, I, 0, 0, 0, nullptr, nullptr, t_given, c_given, alpha,
-                                                               qmax, t, c, a_dev, b_dev, ra_dev, rb_dev, zero_count);
+        k2_scales_from_vectors<<<k2v_blocks, kThreads, 0, st>>>(T, I, t_given, c_given, alpha, qmax, a_dev, b_dev,
+                                                                ra_dev, rb_dev, zero_count);
     } else if (fast_in) {
-        dim3 grid(p.nstrips, p.nrb1);
-        const int64_t cp_ld = static_cast<int64_t>(p.I8) * 8;
+        const int col_ctas = (p.I8 + 31) / 32;
+        const unsigned blocks = static_cast<unsigned>(col_ctas + (T + kThreads - 1) / kThreads);
+        const uint4* cp4 = reinterpret_cast<const uint4*>(colpart);
         if (dtype == CQ_F16) {
-            k1_absmax<false, CQ_F16><<<grid, p.W, 0, st>>>(static_cast<const uint4*>(X), T, p.I8, ld / 8, p.R1, p.nstrips,
-                                                             rowpart, reinterpret_cast<uint4*>(colpart), nullptr, nullptr);
-            k2_scales<CQ_F16><<<k2_blocks, kThreads, 0, st>>>(T, I, p.nstrips, p.nrb1, cp_ld, rowpart, colpart, nullptr,
-                                                              nullptr, alpha, qmax, t_dev, c_dev, a_dev, b_dev, ra_dev,
-                                                              rb_dev, zero_count);
+            const int Y = launch_k1<false, CQ_F16>(p, X, T, ld, rowpart, colpart, nullptr, nullptr, st);
+            launch_dependent(k2_scales_from_partials<CQ_F16>, dim3(blocks), dim3(kThreads), st, T, I, p.I8, p.nstrips, Y,
+                             col_ctas, static_cast<const uint16_t*>(rowpart), cp4, alpha, qmax, t_dev, c_dev, a_dev, b_dev,
+                             ra_dev, rb_dev, zero_count);
         } else {
-            k1_absmax<false, CQ_BF16><<<grid, p.W, 0, st>>>(static_cast<const uint4*>(X), T, p.I8, ld / 8, p.R1, p.nstrips,
-                                                              rowpart, reinterpret_cast<uint4*>(colpart), nullptr, nullptr);
-            k2_scales<CQ_BF16><<<k2_blocks, kThreads, 0, st>>>(T, I, p.nstrips, p.nrb1, cp_ld, rowpart, colpart, nullptr,
-                                                               nullptr, alpha, qmax, t_dev, c_dev, a_dev, b_dev, ra_dev,
-                                                               rb_dev, zero_count);
+            const int Y = launch_k1<false, CQ_BF16>(p, X, T, ld, rowpart, colpart, nullptr, nullptr, st);
+            launch_dependent(k2_scales_from_partials<CQ_BF16>, dim3(blocks), dim3(kThreads), st, T, I, p.I8, p.nstrips, Y,
+                             col_ctas, static_cast<const uint16_t*>(rowpart), cp4, alpha, qmax, t_dev, c_dev, a_dev, b_dev,
+                             ra_dev, rb_dev, zero_count);
         }
     } else {
         rc = absmax_atomic(X, dtype, T, I, ld, t_dev, c_dev, st);
         if (rc != CQ_OK) return rc;
-        if (dtype == CQ_F16)
-            k2_scales<CQ_F16><<<k2_blocks, kThreads, 0, st>>>(T, I, 0, 0, 0, nullptr, nullptr, t_dev, c_dev, alpha, qmax,
-                                                              nullptr, nullptr, a_dev, b_dev, ra_dev, rb_dev, zero_count);
-        else
-            k2_scales<CQ_BF16><<<k2_blocks, kThreads, 0, st>>>(T, I, 0, 0, 0, nullptr, nullptr, t_dev, c_dev, alpha, qmax,
-                                                               nullptr, nullptr, a_dev, b_dev, ra_dev, rb_dev, zero_count);
+        k2_scales_from_vectors<<<k2v_blocks, kThreads, 0, st>>>(T, I, t_dev, c_dev, alpha, qmax, a_dev, b_dev, ra_dev,
+                                                                rb_dev, zero_count);
     }
     if ((rc = launch_status()) != CQ_OK) return rc;
 
@@ -498,16 +722,14 @@ int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
         const bool timed = g_ev_before != nullptr && g_ev_after != nullptr;
         if (timed) cudaEventRecord(g_ev_before, st);
         if (fast_in && fast_out) {
-            dim3 grid(p.nstrips, p.nrb3);
             const int deq_mode = deq == nullptr ? 0 : (deq_dtype == CQ_F32 ? 2 : 1);
-            const uint4* Xv = static_cast<const uint4*>(X);
-            const bool hc = codes != nullptr, hz = zero_count != nullptr;
+            const K3Args k{static_cast<const uint4*>(X), T, p.I8, ld / 8, a_dev, ra_dev, b_dev, rb_dev, codes, deq, zero_count};
             if (dtype == CQ_F16) {
-                if (bits == 8) launch_k3_deq<CQ_F16, 8>(deq_mode, hc, hz, grid, p.W, st, Xv, T, p.I8, ld / 8, p.R3, a_dev, ra_dev, b_dev, rb_dev, codes, deq, zero_count);
-                else launch_k3_deq<CQ_F16, 4>(deq_mode, hc, hz, grid, p.W, st, Xv, T, p.I8, ld / 8, p.R3, a_dev, ra_dev, b_dev, rb_dev, codes, deq, zero_count);
+                if (bits == 8) launch_k3_deq<CQ_F16, 8>(p, k, deq_mode, st);
+                else launch_k3_deq<CQ_F16, 4>(p, k, deq_mode, st);
             } else {
-                if (bits == 8) launch_k3_deq<CQ_BF16, 8>(deq_mode, hc, hz, grid, p.W, st, Xv, T, p.I8, ld / 8, p.R3, a_dev, ra_dev, b_dev, rb_dev, codes, deq, zero_count);
-                else launch_k3_deq<CQ_BF16, 4>(deq_mode, hc, hz, grid, p.W, st, Xv, T, p.I8, ld / 8, p.R3, a_dev, ra_dev, b_dev, rb_dev, codes, deq, zero_count);
+                if (bits == 8) launch_k3_deq<CQ_BF16, 8>(p, k, deq_mode, st);
+                else launch_k3_deq<CQ_BF16, 4>(p, k, deq_mode, st);
             }
         } else {
             const int64_t n = T * ((I + 1) / 2);
@@ -521,6 +743,10 @@ int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
         }
         if (timed) cudaEventRecord(g_ev_after, st);
         if ((rc = launch_status()) != CQ_OK) return rc;
+    }
+    if (c != nullptr && !c_in_place && !given) {
+        if (cudaMemcpyAsync(c, c_dev, sizeof(float) * I, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+            return CQ_ERR_CUDA;
     }
     if (col_scale != nullptr && !b_in_place) {
         if (cudaMemcpyAsync(col_scale, b_dev, sizeof(float) * I, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
@@ -553,11 +779,13 @@ const char* cq_status_string(int status) {
 
 int cq_set_tuning(const char* key, int value) {
     if (key == nullptr) return CQ_ERR_NULL;
-    if (value > cq::kMaxRowsPerCta * 32) return CQ_ERR_SHAPE;
-    const char* k1 = "k1_rows"; const char* k3 = "k3_rows";
+    if (value > 64) return CQ_ERR_SHAPE;
     auto eq = [](const char* x, const char* y) { while (*x && *x == *y) { ++x; ++y; } return *x == *y; };
-    if (eq(key, k1)) { cq::g_tune_k1_rows = value > 0 ? value : 0; return CQ_OK; }
-    if (eq(key, k3)) { cq::g_tune_k3_rows = value > 0 ? value : 0; return CQ_OK; }
+    const int v = value > 0 ? value : 0;
+    if (eq(key, "k1_ctas_per_sm")) { cq::g_tune_k1_ctas = v; return CQ_OK; }
+    if (eq(key, "k3_ctas_per_sm")) { cq::g_tune_k3_ctas = v; return CQ_OK; }
+    if (eq(key, "k3_forward")) { cq::g_tune_k3_forward = v ? 1 : 0; return CQ_OK; }
+    if (eq(key, "no_pdl")) { cq::g_tune_no_pdl = v ? 1 : 0; return CQ_OK; }
     return CQ_ERR_SHAPE;
 }
 

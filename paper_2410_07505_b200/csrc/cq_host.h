@@ -12,9 +12,9 @@ struct Plan {
     int I8;        // vectors of 8 columns per row
     int W;         // threads per CTA = vectors per column strip
     int nstrips;   // column strips
-    int R1, nrb1;  // rows per CTA and row blocks of the absmax pass
-    int R3, nrb3;  // the same for the quantize pass
-    size_t off_t, off_c, off_a, off_b, off_ra, off_rb, off_rowpart, off_colpart, total;
+    int64_t ngroups;  // groups of 4 rows
+    int ycap;      // most CTAs per strip the absmax pass may use (rows of the column-partial buffer)
+    size_t off_t, off_c, off_a, off_b, off_ra, off_rb, off_counters, off_rowpart, off_colpart, total;
 };
 
 Plan make_plan(int64_t T, int64_t I);

@@ -101,7 +101,8 @@ def test_other_entry_points_reject_bad_arguments(lib):
     assert lib.cq_quantize_act_host(FAKE, 1, 4, 8, 8, 0.15, 8, None, None, None, None, None, None, 1, None, None, 0,
                                     None) == 7
     assert lib.cq_set_tuning(b"no_such_knob", 4) == 2
-    assert lib.cq_set_tuning(b"k3_rows", 0) == 0
+    assert lib.cq_set_tuning(b"k3_ctas_per_sm", 0) == 0
+    assert lib.cq_set_tuning(b"k3_ctas_per_sm", 1000) == 2
 
 
 def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):

@@ -152,13 +152,22 @@ def test_tiling_knobs_do_not_change_results(cq):
     X = wl.small_matrix(333, 2304, "bf16", 13, outlier_cols=3)
     ref = orc.quantize_act(X, "bf16", 0.15, 8)
     try:
-        for k1, k3 in [(16, 4), (32, 64), (128, 128), (64, 8)]:
-            cq.set_tuning("k1_rows", k1)
-            cq.set_tuning("k3_rows", k3)
+        for k1, k3, fwd in [(1, 1, 0), (2, 5, 1), (8, 2, 0), (3, 64, 1)]:
+            cq.set_tuning("k1_ctas_per_sm", k1)
+            cq.set_tuning("k3_ctas_per_sm", k3)
+            cq.set_tuning("k3_forward", fwd)
             run_and_check(cq, X, "bf16", 0.15, 8, ref=ref)
     finally:
-        cq.set_tuning("k1_rows", 0)
-        cq.set_tuning("k3_rows", 0)
+        for key in ("k1_ctas_per_sm", "k3_ctas_per_sm", "k3_forward"):
+            cq.set_tuning(key, 0)
+
+
+def test_tall_and_wide_extremes(cq):
+    # many more row groups than resident CTAs, and a single group
+    for T, I in [(5000, 64), (20000, 8), (2, 16384), (4, 40000)]:
+        X = wl.small_matrix(T, I, "f16", 15, outlier_cols=1)
+        run_and_check(cq, X, "f16", 0.15, 8)
+        run_and_check(cq, X, "f16", 0.5, 4)
 
 
 def test_repeated_calls_reuse_buffers(cq):
