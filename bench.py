@@ -42,7 +42,8 @@ HOOK_EVERY = 8
 
 # DRAM traffic of the quantize pass from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum
 # per launch), valid only for the kernel sources whose digest is recorded with it.
-NCU_TRAFFIC = {"sources_sha256": None, "bytes_per_launch": None}
+NCU_TRAFFIC = {"sources_sha256": "0f231ec4fff1c168e931e6345b77cc9484e05f61b23225b346cf92a21f860c20",
+               "bytes_per_launch": 532098048}   # 235,176,192 read + 296,921,856 written
 
 
 def kernel_sources_digest() -> str:
@@ -123,6 +124,21 @@ def rank_config(rank: int):
     if rank:
         cfg = dataclasses.replace(cfg, seed=cfg.seed + 100 * rank)
     return cfg
+
+
+def max_over_ranks(local_ms: float, device: str) -> float:
+    """Largest per-rank device time; every rank gets the same answer (one all-reduce MAX)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([local_ms], dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbs(elements_per_rank: int, steps: int, world: int, max_ms: float) -> float:
+    """Aggregate algorithmic GB/s of `world` independent ranks over the slowest rank's time."""
+    return BYTES_PER_ELEMENT_STEP * elements_per_rank * steps * world / (max_ms * 1e-3) / 1e9
 
 
 def run_reference(args) -> None:
@@ -229,11 +245,8 @@ def main() -> None:
         dist.barrier()
     step_ms = [e[0].elapsed_time(e[1]) for e in ev]
     quant_ms = [ev[k][2].elapsed_time(ev[k][3]) for k in hooked]
-    total_ms = torch.tensor([sum(step_ms)], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(total_ms, op=dist.ReduceOp.MAX)
-    total_ms = float(total_ms.item())
-    value = BYTES_PER_ELEMENT_STEP * n * K * world / (total_ms * 1e-3) / 1e9
+    total_ms = max_over_ranks(sum(step_ms), "cuda")
+    value = whole_job_gbs(n, K, world, total_ms)
     zero_count = int(buf.zero_count.item())
 
     # ---- end to end: host buffers in, host buffers out, through cq_quantize_act_host
@@ -252,10 +265,8 @@ def main() -> None:
         cq.quantize_act_host(Xp, ALPHA, BITS, buffers=hb)
         e1[k].record()
     torch.cuda.synchronize()
-    e2e_ms = torch.tensor([sum(a.elapsed_time(b) for a, b in zip(e0, e1))], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
-    e2e_value = BYTES_PER_ELEMENT_STEP * n * Ke * world / (float(e2e_ms.item()) * 1e-3) / 1e9
+    e2e_ms = max_over_ranks(sum(a.elapsed_time(b) for a, b in zip(e0, e1)), "cuda")
+    e2e_value = whole_job_gbs(n, Ke, world, e2e_ms)
     assert int(hb.zero_count.item()) == zero_count
 
     if rank != 0:
@@ -294,16 +305,16 @@ def main() -> None:
 
     # ---- the oracle on the host cores, bounded sample of the same workload
     from oracle import cq_oracle as orc
-    rows = 1024
-    Xs = X[:rows]
     orc.quantize_act(X[:64], cfg.dtype, ALPHA, BITS, want_deq32=False)
-    t0 = time.perf_counter()
-    orc.quantize_act(Xs, cfg.dtype, ALPHA, BITS, want_deq32=False)
+    reps, t0 = 0, time.perf_counter()
+    while reps < 3 or (time.perf_counter() - t0 < 1.5 and reps < 50):
+        orc.quantize_act(X, cfg.dtype, ALPHA, BITS, want_deq32=False)
+        reps += 1
     dt = time.perf_counter() - t0
-    out["cpu_baseline"] = {"value": BYTES_PER_ELEMENT_STEP * Xs.size / dt / 1e9, "unit": UNIT,
+    out["cpu_baseline"] = {"value": BYTES_PER_ELEMENT_STEP * X.size * reps / dt / 1e9, "unit": UNIT,
                            "cores": orc.num_threads(), "kind": "oracle",
-                           "sample": f"first {rows} rows of the workload matrix ({rows}x{I}), one oracle quantize_act "
-                                     f"(t, c, codes, bf16 dequant, count), {dt:.2f} s"}
+                           "sample": f"the whole workload matrix ({T}x{I}), {reps} oracle quantize_act calls "
+                                     f"(t, c, codes, bf16 dequant, count) in {dt:.2f} s wall on {orc.num_threads()} threads"}
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()

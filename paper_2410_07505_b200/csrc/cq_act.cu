@@ -485,9 +485,9 @@ static cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
 static inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
 // Upper bound on the CTAs per column strip of pass 1 (= rows of the column-partial buffer): keeps
-// that buffer at 8 MiB or less whatever the device.
+// that buffer at 4 MiB or less whatever the device.
 static int y_cap(int I8) {
-    int64_t cap = (int64_t(8) << 20) / (static_cast<int64_t>(I8 > 0 ? I8 : 1) * 16);
+    int64_t cap = (int64_t(4) << 20) / (static_cast<int64_t>(I8 > 0 ? I8 : 1) * 16);
     if (cap < 8) cap = 8;
     if (cap > 2048) cap = 2048;
     return static_cast<int>(cap);
@@ -517,7 +517,6 @@ Plan make_plan(int64_t T, int64_t I) {
     p.off_b = carve(sizeof(float) * static_cast<size_t>(p.I8) * 8);
     p.off_ra = carve(sizeof(float) * static_cast<size_t>(T));
     p.off_rb = carve(sizeof(float) * static_cast<size_t>(p.I8) * 8);
-    p.off_counters = carve(sizeof(unsigned int) * (static_cast<size_t>(p.nstrips) + 65536));
     p.off_rowpart = carve(sizeof(uint16_t) * static_cast<size_t>(T) * p.nstrips);
     const int64_t ymax = p.ngroups < p.ycap ? (p.ngroups > 0 ? p.ngroups : 1) : p.ycap;
     p.off_colpart = carve(sizeof(uint16_t) * static_cast<size_t>(ymax) * static_cast<size_t>(p.I8) * 8);
