@@ -50,7 +50,9 @@ typedef enum {
     CQ_ERR_ALPHA = 5,      /* alpha outside [0, 1] or NaN                                  */
     CQ_ERR_ALIGN = 6,      /* pointer not aligned to its element size, or odd I with INT4  */
     CQ_ERR_WORKSPACE = 7,  /* workspace NULL, misaligned (256 B) or smaller than required  */
-    CQ_ERR_CUDA = 8        /* the CUDA runtime reported an error at launch                 */
+    CQ_ERR_CUDA = 8,       /* the CUDA runtime reported an error at launch                 */
+    CQ_ERR_TOO_LARGE = 9   /* the matrix needs more scratch than the built-in buffer of
+                              cq_quantize_act_noalloc holds                                */
 } cq_status;
 
 typedef enum { CQ_F16 = 0, CQ_BF16 = 1, CQ_F32 = 2 /* outputs only */ } cq_dtype;
@@ -92,6 +94,38 @@ int cq_quantize_act(const void* X, int dtype, int64_t T, int64_t I, int64_t ld,
                     void* codes, void* deq, int deq_dtype,
                     unsigned long long* zero_count,
                     void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * cq_quantize_act for callers that cannot allocate device memory.  (The paper has no counterpart to
+ * this function: it exists for deployment, not for the method.)
+ *
+ * Who needs it: a process that gave the whole GPU to one memory pool at start-up and has no allocator of
+ * its own to ask; a plug-in on a latency-critical path where the host application forbids cudaMalloc
+ * (which synchronises the device and may fail when memory is fragmented); any component whose device
+ * memory budget was fixed before it was loaded.  Such a caller still owns X and every output buffer it
+ * passes, but has nowhere to take the scratch space from that cq_quantize_act asks for.
+ *
+ * Here the scratch is a fixed array of CQ_NOALLOC_SCRATCH_BYTES (8 MiB) inside the library image: every
+ * GPU on which the library is loaded holds that much until the process exits.  Arguments and results
+ * are exactly those of cq_quantize_act without `workspace` / `workspace_bytes`.  The function calls no
+ * cudaMalloc, cudaFree or other allocating routine, on any call.
+ *
+ *   - Limit: shapes with cq_workspace_bytes(T, I) > CQ_NOALLOC_SCRATCH_BYTES return CQ_ERR_TOO_LARGE and
+ *     enqueue nothing.  (4096 x 28672 needs 4.5 MiB; every benchmark configuration fits.)
+ *   - First call on a device: it looks up the array's address on the current device (one
+ *     cudaGetSymbolAddress, remembered afterwards).  Make that first call with the right device current
+ *     and before starting any stream capture.
+ *   - All calls on a device share the one array and find the previous call's contents in it; nothing in
+ *     it needs clearing between calls.  Two calls whose kernels may overlap on the GPU (different
+ *     streams without an ordering between them) race on the array and give undefined results: keep
+ *     calls on one device ordered, e.g. on one stream.
+ */
+#define CQ_NOALLOC_SCRATCH_BYTES (8u << 20)
+int cq_quantize_act_noalloc(const void* X, int dtype, int64_t T, int64_t I, int64_t ld,
+                            double alpha, int bits,
+                            float* t, float* c, float* row_scale, float* col_scale,
+                            void* codes, void* deq, int deq_dtype,
+                            unsigned long long* zero_count, void* stream);
 
 /*
  * Same operation on HOST buffers: copies X to the device, runs cq_quantize_act and copies

@@ -22,7 +22,7 @@ EXPORTS = (
     "cq_version", "cq_status_string", "cq_absmax_rows", "cq_absmax_cols", "cq_absmax_rows_cols",
     "cq_workspace_bytes", "cq_quantize_act", "cq_host_scratch_bytes", "cq_quantize_act_host",
     "cq_dequantize", "cq_kernel_count", "cq_kernel_count_x", "cq_quantize_weight_per_channel",
-    "cq_set_tuning", "cq_set_timing_events",
+    "cq_set_tuning", "cq_set_timing_events", "cq_quantize_act_noalloc",
 )
 
 
@@ -54,6 +54,7 @@ def lib() -> C.CDLL:
         L.cq_workspace_bytes.argtypes = [i64, i64]
         L.cq_quantize_act.argtypes = [vp, ci, i64, i64, i64, dbl, ci, vp, vp, vp, vp, vp, vp, ci, vp, vp,
                                       C.c_size_t, vp]
+        L.cq_quantize_act_noalloc.argtypes = [vp, ci, i64, i64, i64, dbl, ci, vp, vp, vp, vp, vp, vp, ci, vp, vp]
         L.cq_host_scratch_bytes.restype = C.c_size_t
         L.cq_host_scratch_bytes.argtypes = [i64, i64, ci, ci, ci, ci]
         L.cq_quantize_act_host.argtypes = [vp, ci, i64, i64, i64, dbl, ci, vp, vp, vp, vp, vp, vp, ci, vp, vp,
@@ -198,6 +199,25 @@ def quantize_act(X: torch.Tensor, alpha: float = 0.15, bits: int = 8, *, codes: 
                                _ptr(b.row_scale), _ptr(b.col_scale), _ptr(b.codes), _ptr(b.deq), deq_dt,
                                _ptr(b.zero_count), _ptr(b.workspace), b.workspace.numel(), _stream())
     _check(st, "cq_quantize_act")
+    return ActQuant(b.t, b.c, b.row_scale, b.col_scale, b.codes, b.deq, b.zero_count, bits)
+
+
+NOALLOC_SCRATCH_BYTES = 8 << 20
+
+
+def quantize_act_noalloc(X: torch.Tensor, alpha: float = 0.15, bits: int = 8, *, buffers: ActBuffers) -> ActQuant:
+    """quantize_act for callers that cannot allocate device memory: the scratch space is a fixed 8 MiB
+    array inside the library instead of ``buffers.workspace`` (which is not used).  The caller supplies
+    every output through ``buffers``; shapes whose scratch exceeds 8 MiB raise CQError (status 9).  Calls
+    on one device must not overlap on the GPU -- they share the array.  The first call on a device looks
+    the array up and should come before any stream capture."""
+    T, I, ld = _matrix_args(X)
+    b = buffers
+    deq_dt = _DT[b.deq.dtype] if b.deq is not None else _DT[X.dtype]
+    st = lib().cq_quantize_act_noalloc(_ptr(X), _DT[X.dtype], T, I, ld, float(alpha), int(bits), _ptr(b.t), _ptr(b.c),
+                                       _ptr(b.row_scale), _ptr(b.col_scale), _ptr(b.codes), _ptr(b.deq), deq_dt,
+                                       _ptr(b.zero_count), _stream())
+    _check(st, "cq_quantize_act_noalloc")
     return ActQuant(b.t, b.c, b.row_scale, b.col_scale, b.codes, b.deq, b.zero_count, bits)
 
 

@@ -772,6 +772,7 @@ const char* cq_status_string(int status) {
         case CQ_ERR_ALIGN: return "misaligned pointer, or odd number of columns with INT4";
         case CQ_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case CQ_ERR_CUDA: return "CUDA runtime error at launch";
+        case CQ_ERR_TOO_LARGE: return "matrix needs more scratch than the built-in no-allocation buffer holds";
         default: return "unknown status";
     }
 }

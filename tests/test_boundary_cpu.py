@@ -43,8 +43,8 @@ def test_library_exports_every_declared_symbol(lib):
 def test_status_strings(lib):
     from paper_2410_07505_b200 import cq
     assert cq.version() >= 100
-    seen = {cq.status_string(s) for s in range(9)}
-    assert len(seen) == 9 and cq.status_string(0) == "ok"
+    seen = {cq.status_string(s) for s in range(10)}
+    assert len(seen) == 10 and cq.status_string(0) == "ok"
     assert cq.status_string(99) == "unknown status"
 
 
@@ -100,6 +100,9 @@ def test_other_entry_points_reject_bad_arguments(lib):
     assert lib.cq_quantize_weight_per_channel(None, 1, 4, 8, 8, 8, FAKE, FAKE, None, 1, None, None) == 1
     assert lib.cq_quantize_act_host(FAKE, 1, 4, 8, 8, 0.15, 8, None, None, None, None, None, None, 1, None, None, 0,
                                     None) == 7
+    # far beyond the built-in scratch of the no-allocation entry point: refused before any CUDA call
+    assert lib.cq_quantize_act_noalloc(FAKE, 1, 1 << 24, 4096, 4096, 0.15, 8, None, None, None, None, FAKE, None, 1,
+                                       None, None) == 9
     assert lib.cq_set_tuning(b"no_such_knob", 4) == 2
     assert lib.cq_set_tuning(b"k3_ctas_per_sm", 0) == 0
     assert lib.cq_set_tuning(b"k3_ctas_per_sm", 1000) == 2
