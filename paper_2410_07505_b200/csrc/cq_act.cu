@@ -26,14 +26,14 @@ __device__ __forceinline__ void row_scale_of(float ti, double alpha, int qmax, f
     if (alpha == 1.0) ai = __fdiv_rn(ti, static_cast<float>(qmax));
     else if (alpha == 0.0) ai = 1.0f;
     else ai = static_cast<float>(pow(static_cast<double>(ti), alpha) / static_cast<double>(qmax));
-    rai = __fdiv_rn(1.0f, ai);
+    rai = guarded_rcp(ai);
 }
 
 __device__ __forceinline__ void col_scale_of(float cj, double alpha, int qmax, float& bj, float& rbj) {
     if (alpha == 1.0) bj = 1.0f;
     else if (alpha == 0.0) bj = __fdiv_rn(cj, static_cast<float>(qmax));
     else bj = static_cast<float>(pow(static_cast<double>(cj), 1.0 - alpha));
-    rbj = __fdiv_rn(1.0f, bj);
+    rbj = guarded_rcp(bj);
 }
 
 // ============================================================================ pass 1: absmax
@@ -257,63 +257,6 @@ k2_scales_from_vectors(int64_t T, int64_t I, const float* __restrict__ t_in, con
 }
 
 // ============================================================================ pass 2: quantize
-// Outside [2^-60, 2^60] a scale factor or its reciprocal may have lost relative precision (fp32
-// subnormals); such rows and columns are never trusted to the candidate test.
-constexpr float kScaleLo = 8.6736173798840355e-19f;    // 2^-60
-constexpr float kScaleHi = 1.152921504606846976e18f;   // 2^60
-// The candidate q = round-half-even(v), v = x * (1/a_i) * (1/b_j), is accepted when |v - q| < 1/2 - 2^-12.
-// With a_i, b_j, their reciprocals and s_ij all normal, v differs from z = x / s_ij by less than
-// 5 * 2^-24 |z| <= 2^-14.6 (|z| <= 128), so |z - q| < 1/2 - 2^-12 + 2^-14.6 and the IEEE quotient
-// fl32(z), which lies within 2^-17 of z, rounds to the same q; |z| <= qmax (1 + 2^-22) keeps q in range.
-constexpr float kAcceptBelow = 0.499755859375f;         // 1/2 - 2^-12
-
-// Eight elements of one row in packed fp32x2 arithmetic (bit-identical to the scalar IEEE operations,
-// half the issue slots).  y2[k] = kMagic + q and q2[k] = q for elements 2k, 2k+1.
-template <int DT, int BITS>
-__device__ __forceinline__ void quantize_row8(const uint4& w, float a, float ra, const float2 (&b2)[4],
-                                              const float2 (&rb2)[4], bool row_safe,
-                                              float2 (&y2)[4], float2 (&q2)[4]) {
-    constexpr float qmaxf = static_cast<float>((1 << (BITS - 1)) - 1);
-    const float2 ra2 = make_float2(ra, ra);
-    const float2 m2 = make_float2(kMagic, kMagic), nm2 = make_float2(-kMagic, -kMagic);
-    const float2 neg1 = make_float2(-1.0f, -1.0f);
-    const uint32_t words[4] = {w.x, w.y, w.z, w.w};
-    float worst = 0.0f;
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        const float2 x = unpack16x2<DT>(words[k]);
-        const float2 r = __fmul2_rn(ra2, rb2[k]);
-        const float2 v = __fmul2_rn(x, r);                    // x / s, approximately
-        y2[k] = __fadd2_rn(v, m2);
-        q2[k] = __fadd2_rn(y2[k], nm2);                       // round-half-even(v), exact
-        const float2 f = __ffma2_rn(q2[k], neg1, v);          // v - q, exact
-        worst = fmaxf(fmaxf(worst, fabsf(f.x)), fabsf(f.y));
-    }
-    if (!(row_safe && worst < kAcceptBelow)) {
-        // Rare: some element is too close to a rounding boundary (or a scale is extreme / zero / NaN)
-        // for the cheap test to decide.  Re-examine each element with the exact residual; the
-        // undecided ones take the defining sequence (IEEE division, round half to even, clamp).
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const float2 x = unpack16x2<DT>(words[k]);
-            const float xs[2] = {x.x, x.y};
-            const float bs[2] = {b2[k].x, b2[k].y};
-            const float rs[2] = {rb2[k].x, rb2[k].y};
-            float ys[2];
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const float sh = __fmul_rn(a, bs[h]);
-                bool good;
-                ys[h] = quant_candidate(xs[h], sh, __fmul_rn(ra, rs[h]), qmaxf, good);
-                good = good && a >= kScaleLo && bs[h] >= kScaleLo && sh >= kScaleLo;
-                if (!good) ys[h] = quant_exact(xs[h], sh, qmaxf);
-            }
-            y2[k] = make_float2(ys[0], ys[1]);
-            q2[k] = __fadd2_rn(y2[k], nm2);
-        }
-    }
-}
-
 // Same strip / resident-CTA layout and rolling four-row prefetch as pass 1.  Full row groups are
 // walked from the last one backwards (the rows pass 1 touched last are the likeliest to be still in
 // L2) unless `forward` is set; a ragged last group (T not a multiple of 4) is done first by CTA y = 0.
@@ -340,7 +283,6 @@ k3_quantize(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
 
     if (warp_active) {
         float2 b2[4], rb2[4];
-        float bmin;
         {
             const float4* bp = reinterpret_cast<const float4*>(b) + static_cast<int64_t>(vv) * 2;
             const float4* rp = reinterpret_cast<const float4*>(rb) + static_cast<int64_t>(vv) * 2;
@@ -349,25 +291,25 @@ k3_quantize(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
             b2[2] = make_float2(b1.x, b1.y); b2[3] = make_float2(b1.z, b1.w);
             rb2[0] = make_float2(q0.x, q0.y); rb2[1] = make_float2(q0.z, q0.w);
             rb2[2] = make_float2(q1.x, q1.y); rb2[3] = make_float2(q1.z, q1.w);
-            bmin = fminf(fminf(fminf(b0.x, b0.y), fminf(b0.z, b0.w)), fminf(fminf(b1.x, b1.y), fminf(b1.z, b1.w)));
-            const float bmax = fmaxf(fmaxf(fmaxf(b0.x, b0.y), fmaxf(b0.z, b0.w)), fmaxf(fmaxf(b1.x, b1.y), fmaxf(b1.z, b1.w)));
-            if (!(bmin >= kScaleLo && bmax <= kScaleHi)) bmin = 0.0f;      // never trust this thread's columns
         }
+        // false if any of this thread's eight column reciprocals is the NaN marker of an extreme scale
+        const bool cols_trusted = ((rb2[0].x + rb2[0].y) + (rb2[1].x + rb2[1].y)) +
+                                  ((rb2[2].x + rb2[2].y) + (rb2[3].x + rb2[3].y)) < INFINITY;
         const uint4* xp = X + vv;
 
-        // one row of 8 elements: quantize, pack, store (stores only from lanes that own a column)
-        auto do_row = [&](const uint4& wrow, float au, float rau, int64_t vec) {
-            const bool row_safe = au >= kScaleLo && au <= kScaleHi && __fmul_rn(au, bmin) >= kScaleLo;
+        // One row of 8 elements: quantize, re-load the row slot for the next group, pack, store
+        // (stores only from lanes that own a column).  `vec` indexes 8-element vectors of the outputs.
+        auto do_row = [&](uint4& slot, const uint4* reload, bool has_next, float au, float rau, int vec) {
             float2 y2[4], q2[4];
-            quantize_row8<DT, BITS>(wrow, au, rau, b2, rb2, row_safe, y2, q2);
+            quantize_row8<DT, BITS, false>(slot, au, rau, b2, rb2, cols_trusted && rau == rau, y2, q2);
+            if (has_next) slot = ld_stream(reload);
             if constexpr (BITS == 8) {
                 const uint32_t c0 = pack_int8x4(y2[0].x, y2[0].y, y2[1].x, y2[1].y);
                 const uint32_t c1 = pack_int8x4(y2[2].x, y2[2].y, y2[3].x, y2[3].y);
                 if constexpr (COUNT) zeros += zero_bytes(c0) + zero_bytes(c1);
                 if constexpr (CODES) { if (active) st_stream(reinterpret_cast<uint2*>(codes) + vec, make_uint2(c0, c1)); }
             } else {
-                const float ys[8] = {y2[0].x, y2[0].y, y2[1].x, y2[1].y, y2[2].x, y2[2].y, y2[3].x, y2[3].y};
-                const uint32_t c0 = pack_int4x8(ys);
+                const uint32_t c0 = pack_int4x8(y2);
                 if constexpr (COUNT) zeros += zero_nibbles(c0);
                 if constexpr (CODES) { if (active) st_stream(reinterpret_cast<uint32_t*>(codes) + vec, c0); }
             }
@@ -382,7 +324,7 @@ k3_quantize(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
                     o.z = pack16x2<DT>(d2[2].x, d2[2].y); o.w = pack16x2<DT>(d2[3].x, d2[3].y);
                     if (active) st_stream(reinterpret_cast<uint4*>(deq) + vec, o);
                 } else {
-                    float4* o = reinterpret_cast<float4*>(deq) + vec * 2;
+                    float4* o = reinterpret_cast<float4*>(deq) + static_cast<int64_t>(vec) * 2;
                     if (active) {
                         st_stream(o, make_float4(d2[0].x, d2[0].y, d2[1].x, d2[1].y));
                         st_stream(o + 1, make_float4(d2[2].x, d2[2].y, d2[3].x, d2[3].y));
@@ -400,8 +342,9 @@ k3_quantize(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
             const float arv = load_scales(nfull);
             for (int u = 0; u < static_cast<int>(T & 3); ++u) {
                 const int64_t row = (nfull << 2) + u;
-                const uint4 wrow = ld_stream(xp + row * ld8);
-                do_row(wrow, __shfl_sync(0xFFFFFFFFu, arv, u), __shfl_sync(0xFFFFFFFFu, arv, 4 + u), row * I8 + vv);
+                uint4 slot = ld_stream(xp + row * ld8);
+                do_row(slot, nullptr, false, __shfl_sync(0xFFFFFFFFu, arv, u), __shfl_sync(0xFFFFFFFFu, arv, 4 + u),
+                       static_cast<int>(row * I8 + vv));
             }
         }
 
@@ -409,9 +352,10 @@ k3_quantize(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
         if (pos < nfull) {
             const int64_t dgroups = forward ? Y : -Y;
             int64_t g = forward ? pos : nfull - 1 - pos;
-            const int64_t xstep = 4 * dgroups * ld8, ostep = 4 * dgroups * static_cast<int64_t>(I8);
+            const int64_t xstep = 4 * dgroups * ld8;
+            const int ostep = static_cast<int>(4 * dgroups * I8);
             const uint4* p = xp + (g << 2) * ld8;
-            int64_t vec = (g << 2) * I8 + vv;
+            int vec = static_cast<int>((g << 2) * I8 + vv);
             uint4 w[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u) w[u] = ld_stream(p + u * ld8);
@@ -422,12 +366,9 @@ k3_quantize(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
                 float arvn = 0.0f;
                 if (has_next) arvn = load_scales(g + dgroups);
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const uint4 cur = w[u];
-                    if (has_next) w[u] = ld_stream(pn + u * ld8);
-                    do_row(cur, __shfl_sync(0xFFFFFFFFu, arv, u), __shfl_sync(0xFFFFFFFFu, arv, 4 + u),
-                           vec + static_cast<int64_t>(u) * I8);
-                }
+                for (int u = 0; u < 4; ++u)
+                    do_row(w[u], pn + u * ld8, has_next, __shfl_sync(0xFFFFFFFFu, arv, u),
+                           __shfl_sync(0xFFFFFFFFu, arv, 4 + u), vec + u * I8);
                 p = pn;
                 vec += ostep;
                 g += dgroups;
@@ -685,7 +626,8 @@ int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
 
     const bool fast_in = fast_input(X, I, ld);
     const bool fast_out = (codes == nullptr || aligned(codes, bits == 8 ? 8 : 4)) &&
-                          (deq == nullptr || aligned(deq, 16));
+                          (deq == nullptr || aligned(deq, 16)) &&
+                          T * static_cast<int64_t>(p.I8) < (int64_t(1) << 31);     // 32-bit vector indices
     const unsigned k2v_blocks = static_cast<unsigned>((T + I + kThreads - 1) / kThreads);
 
     // ---- pass 1 + scale vectors

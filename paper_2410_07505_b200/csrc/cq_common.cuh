@@ -104,6 +104,72 @@ static __device__ __noinline__ float quant_exact(float x, float s, float qmaxf) 
     return __fadd_rn(q, kMagic);        // (-0) + kMagic == kMagic
 }
 
+// ---- eight elements of one row -------------------------------------------------------------
+// Scale factors outside [2^-40, 2^40] get a NaN "reciprocal"; callers test for it (x != x) and send
+// such rows / columns to the defining sequence.  A factor of exactly zero means the whole row or
+// column is zero (t_i = 0 or c_j = 0), so its elements are zeros and any finite reciprocal gives the
+// right candidate, code 0: it gets 0.
+constexpr float kScaleLo = 9.094947017729282e-13f;     // 2^-40
+constexpr float kScaleHi = 1.099511627776e12f;         // 2^40
+__device__ __forceinline__ float guarded_rcp(float f) {
+    if (f == 0.0f) return 0.0f;
+    return (f >= kScaleLo && f <= kScaleHi) ? __fdiv_rn(1.0f, f) : __int_as_float(0x7FC00000);
+}
+// The candidate q = round-half-even(v), v = x * (1/a_i) * (1/b_j), is accepted when |v - q| < 1/2 - 2^-12.
+// With a_i, b_j in [2^-40, 2^40] they, their reciprocals, s_ij = fl32(a_i b_j) and the reciprocal product
+// are all normal numbers, so v differs from z = x / s_ij by less than 5 * 2^-24 |z| <= 2^-14.6 (|z| <= 128);
+// hence |z - q| < 1/2 - 2^-12 + 2^-14.6 and the IEEE quotient fl32(z), which lies within 2^-17 of z, rounds
+// to the same q.  |x| <= min(t_i, c_j) gives |z| <= qmax (1 + 2^-22), which keeps q within [-qmax, qmax].
+constexpr float kAcceptBelow = 0.499755859375f;         // 1/2 - 2^-12
+
+// Packed fp32x2 arithmetic (bit-identical to the scalar IEEE operations, half the issue slots).
+// y2[k] = kMagic + q and q2[k] = q for elements 2k, 2k+1.  UNIFORM: one scale `a` for the whole row
+// (b2, rb2 unused).  `trusted`: none of the reciprocals involved is the NaN marker (a NaN would not
+// survive the max below, so it has to be tested where the reciprocals are loaded).
+template <int DT, int BITS, bool UNIFORM>
+__device__ __forceinline__ void quantize_row8(const uint4& w, float a, float ra, const float2 (&b2)[4],
+                                              const float2 (&rb2)[4], bool trusted,
+                                              float2 (&y2)[4], float2 (&q2)[4]) {
+    constexpr float qmaxf = static_cast<float>((1 << (BITS - 1)) - 1);
+    const float2 ra2 = make_float2(ra, ra);
+    const float2 m2 = make_float2(kMagic, kMagic), nm2 = make_float2(-kMagic, -kMagic);
+    const float2 neg1 = make_float2(-1.0f, -1.0f);
+    const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+    float worst = 0.0f;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const float2 x = unpack16x2<DT>(words[k]);
+        const float2 r = UNIFORM ? ra2 : __fmul2_rn(ra2, rb2[k]);
+        const float2 v = __fmul2_rn(x, r);                    // x / s, approximately
+        y2[k] = __fadd2_rn(v, m2);
+        q2[k] = __fadd2_rn(y2[k], nm2);                       // round-half-even(v), exact
+        const float2 f = __ffma2_rn(q2[k], neg1, v);          // v - q, exact
+        worst = fmaxf(fmaxf(worst, fabsf(f.x)), fabsf(f.y));
+    }
+    if (!(trusted && worst < kAcceptBelow)) {
+        // Rare: some element is too close to a rounding boundary (or a scale factor is extreme) for the
+        // cheap test to decide.  Re-examine each element with the exact residual; the undecided ones
+        // take the defining sequence (IEEE division, round half to even, clamp).
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float2 x = unpack16x2<DT>(words[k]);
+            const float xs[2] = {x.x, x.y};
+            const float bs[2] = {UNIFORM ? 1.0f : b2[k].x, UNIFORM ? 1.0f : b2[k].y};
+            const float rs[2] = {UNIFORM ? 1.0f : rb2[k].x, UNIFORM ? 1.0f : rb2[k].y};
+            float ys[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const float sh = UNIFORM ? a : __fmul_rn(a, bs[h]);
+                bool good;
+                ys[h] = quant_candidate(xs[h], sh, UNIFORM ? ra : __fmul_rn(ra, rs[h]), qmaxf, good);
+                if (!good) ys[h] = quant_exact(xs[h], sh, qmaxf);
+            }
+            y2[k] = make_float2(ys[0], ys[1]);
+            q2[k] = __fadd2_rn(y2[k], nm2);
+        }
+    }
+}
+
 __device__ __forceinline__ float code_as_float(float y) { return __fadd_rn(y, -kMagic); }
 __device__ __forceinline__ int code_as_int(float y) {
     return static_cast<int>(__float_as_uint(y)) - static_cast<int>(kMagicBits);
@@ -116,12 +182,15 @@ __device__ __forceinline__ uint32_t pack_int8x4(float y0, float y1, float y2, fl
     return __byte_perm(p01, p23, 0x5410);
 }
 
-// eight codes -> one word of two's-complement nibbles, element e in bits [4e, 4e+4)
-__device__ __forceinline__ uint32_t pack_int4x8(const float (&y)[8]) {
-    uint32_t w = 0;
+// eight codes -> one word of two's-complement nibbles, element e in bits [4e, 4e+4): each pair of
+// magic-biased floats gives one byte (low nibble | high nibble << 4), the four bytes are then gathered
+__device__ __forceinline__ uint32_t pack_int4x8(const float2 (&y2)[4]) {
+    uint32_t t[4];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) w |= (__float_as_uint(y[e]) & 0xFu) << (4 * e);
-    return w;
+    for (int k = 0; k < 4; ++k) t[k] = (__float_as_uint(y2[k].x) & 0xFu) + __float_as_uint(y2[k].y) * 16u;
+    const uint32_t p01 = __byte_perm(t[0], t[1], 0x0040);
+    const uint32_t p23 = __byte_perm(t[2], t[3], 0x0040);
+    return __byte_perm(p01, p23, 0x5410);
 }
 
 __device__ __forceinline__ int zero_bytes(uint32_t w) {

@@ -37,55 +37,40 @@ k4_weight_rows(const uint4* __restrict__ W, int C8, int64_t ld8,
 #pragma unroll
     for (int k = 0; k < kThreads / 32; ++k) m16 = max(m16, s_max[k]);
     const float d = __fdiv_rn(cvt16<DT>(static_cast<uint16_t>(m16)), qmaxf);
-    const float rd = __fdiv_rn(1.0f, d);
+    const float rd = guarded_rcp(d);
     if (tid == 0 && scale != nullptr) scale[row] = d;
 
+    const float2 ones[4] = {make_float2(1.0f, 1.0f), make_float2(1.0f, 1.0f), make_float2(1.0f, 1.0f), make_float2(1.0f, 1.0f)};
+    const float2 d2s = make_float2(d, d);
     unsigned int zeros = 0;
     for (int v = tid; v < C8; v += kThreads) {
         const uint4 w = s_vec[v];
-        const uint32_t words[4] = {w.x, w.y, w.z, w.w};
-        float x[8], y[8];
-        unsigned int bad = 0;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            float2 f = unpack16x2<DT>(words[k]);
-            x[2 * k] = f.x; x[2 * k + 1] = f.y;
-        }
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            bool ok;
-            y[e] = quant_candidate(x[e], d, rd, qmaxf, ok);
-            bad |= (ok ? 0u : 1u) << e;
-        }
-        if (bad) {
-#pragma unroll
-            for (int e = 0; e < 8; ++e)
-                if ((bad >> e) & 1u) y[e] = quant_exact(x[e], d, qmaxf);
-        }
+        float2 y2[4], q2[4];
+        quantize_row8<DT, BITS, true>(w, d, rd, ones, ones, rd == rd, y2, q2);
         const int64_t vec = row * C8 + v;
         if constexpr (BITS == 8) {
-            uint32_t c0 = pack_int8x4(y[0], y[1], y[2], y[3]);
-            uint32_t c1 = pack_int8x4(y[4], y[5], y[6], y[7]);
+            const uint32_t c0 = pack_int8x4(y2[0].x, y2[0].y, y2[1].x, y2[1].y);
+            const uint32_t c1 = pack_int8x4(y2[2].x, y2[2].y, y2[3].x, y2[3].y);
             zeros += zero_bytes(c0) + zero_bytes(c1);
             if constexpr (CODES) st_stream(reinterpret_cast<uint2*>(codes) + vec, make_uint2(c0, c1));
         } else {
-            uint32_t c0 = pack_int4x8(y);
+            const uint32_t c0 = pack_int4x8(y2);
             zeros += zero_nibbles(c0);
             if constexpr (CODES) st_stream(reinterpret_cast<uint32_t*>(codes) + vec, c0);
         }
         if constexpr (DEQ != 0) {
-            float dq[8];
+            float2 dq[4];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) dq[e] = __fmul_rn(code_as_float(y[e]), d);
+            for (int k = 0; k < 4; ++k) dq[k] = __fmul2_rn(q2[k], d2s);
             if constexpr (DEQ == 1) {
                 uint4 o;
-                o.x = pack16x2<DT>(dq[0], dq[1]); o.y = pack16x2<DT>(dq[2], dq[3]);
-                o.z = pack16x2<DT>(dq[4], dq[5]); o.w = pack16x2<DT>(dq[6], dq[7]);
+                o.x = pack16x2<DT>(dq[0].x, dq[0].y); o.y = pack16x2<DT>(dq[1].x, dq[1].y);
+                o.z = pack16x2<DT>(dq[2].x, dq[2].y); o.w = pack16x2<DT>(dq[3].x, dq[3].y);
                 st_stream(reinterpret_cast<uint4*>(deq) + vec, o);
             } else {
                 float4* o = reinterpret_cast<float4*>(deq) + vec * 2;
-                st_stream(o, make_float4(dq[0], dq[1], dq[2], dq[3]));
-                st_stream(o + 1, make_float4(dq[4], dq[5], dq[6], dq[7]));
+                st_stream(o, make_float4(dq[0].x, dq[0].y, dq[1].x, dq[1].y));
+                st_stream(o + 1, make_float4(dq[2].x, dq[2].y, dq[3].x, dq[3].y));
             }
         }
     }

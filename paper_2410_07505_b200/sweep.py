@@ -1,0 +1,118 @@
+"""Per-configuration timing table and the 80-layer LLaMA-70B-shaped sweep.
+
+    python -m paper_2410_07505_b200.sweep                 # every activation config x bit width, 3 weight shapes
+    python -m paper_2410_07505_b200.sweep --layers 80     # plus the per-layer sweep (inputs generated per layer)
+
+Times are CUDA-event medians of the public calls with the L2 flushed before every call (a 256 MiB
+write) and also back to back without the flush.  GB/s uses the algorithmic byte counts: activations
+2+2+codes+2 bytes per element (X read twice), weights 2+codes+2 (row read once).  One JSON object per line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import statistics
+
+import numpy as np
+import torch
+
+from . import cq
+from . import workloads as wl
+
+TORCH_DT = {"f16": torch.float16, "bf16": torch.bfloat16}
+
+
+def _dev(bits: np.ndarray, dtype: str) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(TORCH_DT[dtype]).cuda()
+
+
+def _time(fn, flush, iters: int) -> float:
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    for a, b in ev:
+        if flush is not None:
+            flush.zero_()
+        a.record()
+        fn()
+        b.record()
+    torch.cuda.synchronize()
+    return statistics.median(a.elapsed_time(b) for a, b in ev) * 1e3     # microseconds
+
+
+def time_activation(Xd: torch.Tensor, bits: int, alpha: float, flush, iters: int) -> dict:
+    T, I = Xd.shape
+    buf = cq.ActBuffers(T, I, Xd.dtype, bits)
+    us_cold = _time(lambda: cq.quantize_act(Xd, alpha, bits, buffers=buf), flush, iters)
+    us_warm = _time(lambda: cq.quantize_act(Xd, alpha, bits, buffers=buf), None, iters)
+    n = T * I
+    per_elem = 2 + 2 + (1 if bits == 8 else 0.5) + 2
+    return {"us_l2_flushed": round(us_cold, 1), "us_back_to_back": round(us_warm, 1),
+            "gbs_l2_flushed": round(per_elem * n / us_cold / 1e3, 1),
+            "gbs_single_read_accounting": round((per_elem - 2) * n / us_cold / 1e3, 1),
+            "elements_per_s": round(n / us_cold * 1e6), "kernel_proportion": int(buf.zero_count.item()) / n}
+
+
+def time_weight(Wd: torch.Tensor, bits: int, flush, iters: int) -> dict:
+    out = cq.quantize_weight_per_channel(Wd, bits)
+    us = _time(lambda: cq.quantize_weight_per_channel(Wd, bits, out=out), flush, iters)
+    n = Wd.numel()
+    per_elem = 2 + (1 if bits == 8 else 0.5) + 2
+    return {"us_l2_flushed": round(us, 1), "gbs": round(per_elem * n / us / 1e3, 1),
+            "kernel_proportion": int(out.zero_count.item()) / n}
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--iters", type=int, default=30)
+    ap.add_argument("--layers", type=int, default=0, help="layers of the 80-layer sweep to run (0 = skip)")
+    ap.add_argument("--alpha", type=float, default=0.15)
+    args = ap.parse_args()
+    cq.lib()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    for name, cfg in wl.ACT_CONFIGS.items():
+        Xd = _dev(wl.generate_activation(cfg), cfg.dtype)
+        for bits in cfg.bits:
+            for alpha in cfg.alphas:
+                row = {"config": name, "shape": [cfg.T, cfg.I], "dtype": cfg.dtype, "bits": bits, "alpha": alpha}
+                row.update(time_activation(Xd, bits, alpha, flush, args.iters))
+                print(json.dumps(row), flush=True)
+        del Xd
+    for k, shape in enumerate(wl.SWEEP_WEIGHT_SHAPES):
+        Wd = _dev(wl.sweep_weight(0, k), "bf16")
+        for bits in (8, 4):
+            row = {"config": f"weight_{shape[0]}x{shape[1]}", "shape": list(shape), "dtype": "bf16", "bits": bits}
+            row.update(time_weight(Wd, bits, flush, args.iters))
+            print(json.dumps(row), flush=True)
+        del Wd
+
+    total_us = 0.0
+    for layer in range(args.layers):
+        props = []
+        layer_us = 0.0
+        for k in range(4):
+            cfg = wl.sweep_activation_config(layer, k)
+            Xd = _dev(wl.generate_activation(cfg), cfg.dtype)
+            for bits in (8, 4):
+                r = time_activation(Xd, bits, args.alpha, flush, max(5, args.iters // 3))
+                layer_us += r["us_l2_flushed"]
+                if bits == 8:
+                    props.append(r["kernel_proportion"])
+            del Xd
+        for k in range(3):
+            Wd = _dev(wl.sweep_weight(layer, k), "bf16")
+            for bits in (8, 4):
+                layer_us += time_weight(Wd, bits, flush, max(5, args.iters // 3))["us_l2_flushed"]
+            del Wd
+        total_us += layer_us
+        print(json.dumps({"layer": layer, "quantizer_us": round(layer_us, 1),
+                          "kernel_proportion_int8_mean": sum(props) / len(props),
+                          "kernel_proportion_int8_each": props}), flush=True)
+    if args.layers:
+        print(json.dumps({"layers": args.layers, "end_to_end_quantizer_ms": round(total_us / 1e3, 3)}))
+
+
+if __name__ == "__main__":
+    main()
