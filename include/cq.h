@@ -172,6 +172,17 @@ int cq_quantize_weight_per_channel(const void* W, int dtype, int64_t R, int64_t 
                                    void* codes, float* scale, void* deq, int deq_dtype,
                                    unsigned long long* zero_count, void* stream);
 
+/*
+ * Group-wise weight quantization (Section 3: W is reshaped to (elements / g) x g and then quantized per
+ * row as in Eq. 2; g = 128 in the paper's W4A8-g128 experiments).  `group` must divide C, so every group
+ * lies inside one stored row; groups are numbered row by row.
+ *   scale out float[R * C / group]; codes / deq as in cq_quantize_weight_per_channel (dense [R x C]).
+ * One read of W for group sizes 8..256 that are powers of two; other sizes take a slower general kernel.
+ */
+int cq_quantize_weight_groupwise(const void* W, int dtype, int64_t R, int64_t C, int64_t ld, int64_t group, int bits,
+                                 void* codes, float* scale, void* deq, int deq_dtype,
+                                 unsigned long long* zero_count, void* stream);
+
 /* Launch-shape knobs for measurement.  key: "k1_ctas_per_sm", "k3_ctas_per_sm" (resident CTAs per SM
  * the two passes size their grids for; 1..64), "k3_forward" (1: the quantize pass walks the rows in
  * ascending order) or "no_pdl" (1: launch the quantize pass without programmatic dependent launch).  value <= 0 restores the built-in choice.  Results never depend on these.

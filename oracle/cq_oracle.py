@@ -191,3 +191,14 @@ def compare_with_ideal(X: np.ndarray, dtype: str, alpha: float, bits: int, res: 
                                  C.c_int(bits), _p(res.t), _p(res.c), _p(res.a), _p(res.b),
                                  _p(np.ascontiguousarray(res.codes)), C.c_double(rel), _p(out))
     return int(out[0]), int(out[1]), int(out[2])
+
+
+def quantize_weight_groupwise(W: np.ndarray, dtype: str, bits: int, group: int) -> WeightResult:
+    """Group-wise weight quantization exactly as the paper states it (Section 3): reshape the weight
+    matrix to (elements / g) x g, quantize per row (Eq. 2), reshape back."""
+    R, Cc = W.shape
+    if group <= 0 or Cc % group:
+        raise ValueError("the group size must divide the number of columns")
+    flat = np.ascontiguousarray(W).reshape(R * Cc // group, group)
+    r = quantize_weight_per_channel(flat, dtype, bits)
+    return WeightResult(r.scale, r.codes.reshape(R, Cc), r.deq32.reshape(R, Cc), r.deq16.reshape(R, Cc), r.zero_count)

@@ -23,6 +23,7 @@ EXPORTS = (
     "cq_workspace_bytes", "cq_quantize_act", "cq_host_scratch_bytes", "cq_quantize_act_host",
     "cq_dequantize", "cq_kernel_count", "cq_kernel_count_x", "cq_quantize_weight_per_channel",
     "cq_set_tuning", "cq_set_timing_events", "cq_quantize_act_noalloc",
+    "cq_quantize_weight_groupwise",
 )
 
 
@@ -63,6 +64,7 @@ def lib() -> C.CDLL:
         L.cq_kernel_count.argtypes = [vp, ci, i64, i64, vp, vp]
         L.cq_kernel_count_x.argtypes = [vp, ci, i64, i64, i64, dbl, ci, vp, vp, vp, vp, C.c_size_t, vp]
         L.cq_quantize_weight_per_channel.argtypes = [vp, ci, i64, i64, i64, ci, vp, vp, vp, ci, vp, vp]
+        L.cq_quantize_weight_groupwise.argtypes = [vp, ci, i64, i64, i64, i64, ci, vp, vp, vp, ci, vp, vp]
         L.cq_set_tuning.argtypes = [C.c_char_p, ci]
         L.cq_set_timing_events.argtypes = [vp, vp]
         for name in EXPORTS:
@@ -321,4 +323,27 @@ def quantize_weight_per_channel(W: torch.Tensor, bits: int = 8, *, codes: bool =
                                               _ptr(out.scale), _ptr(out.deq), deq_dt, _ptr(out.zero_count),
                                               _stream())
     _check(st, "cq_quantize_weight_per_channel")
+    return out
+
+
+def quantize_weight_groupwise(W: torch.Tensor, group: int = 128, bits: int = 4, *, codes: bool = True, deq: bool = True,
+                              deq_dtype: torch.dtype | None = None, count: bool = True,
+                              out: WeightQuant | None = None) -> WeightQuant:
+    """Group-wise weight quantization: every run of ``group`` consecutive elements of a stored row gets
+    its own scale (``out.scale`` has R * C / group entries, row by row)."""
+    R, Cc, ld = _matrix_args(W)
+    if out is None:
+        dev = W.device
+        codes_t = None
+        if codes:
+            codes_t = (torch.empty((R, Cc), dtype=torch.int8, device=dev) if bits == 8
+                       else torch.empty((R, Cc // 2), dtype=torch.uint8, device=dev))
+        n_groups = R * (Cc // group) if group > 0 else 0
+        out = WeightQuant(torch.empty(n_groups, dtype=torch.float32, device=dev), codes_t,
+                          torch.empty((R, Cc), dtype=deq_dtype or W.dtype, device=dev) if deq else None,
+                          torch.zeros((), dtype=torch.int64, device=dev) if count else None, bits)
+    deq_dt = _DT[out.deq.dtype] if out.deq is not None else _DT[W.dtype]
+    st = lib().cq_quantize_weight_groupwise(_ptr(W), _DT[W.dtype], R, Cc, ld, int(group), int(bits), _ptr(out.codes),
+                                            _ptr(out.scale), _ptr(out.deq), deq_dt, _ptr(out.zero_count), _stream())
+    _check(st, "cq_quantize_weight_groupwise")
     return out

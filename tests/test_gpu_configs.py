@@ -72,3 +72,14 @@ def test_sweep_layer_weights(cq, k):
         parity.check_weight(W, "bf16", bits, scale=r.scale.cpu().numpy(), codes=r.codes.cpu().numpy(),
                             deq=bits_of(r.deq), zero_count=int(r.zero_count.item()), ref=ref)
         del r
+
+
+def test_sweep_weight_groupwise_g128(cq):
+    """W4-g128 on a full-size sweep weight (the paper's W4A8-g128 setting)."""
+    W = wl.sweep_weight(0, 1)
+    Wd = to_dev(W, "bf16")
+    ref = orc.quantize_weight_groupwise(W, "bf16", 4, 128)
+    r = cq.quantize_weight_groupwise(Wd, 128, 4)
+    torch.cuda.synchronize()
+    parity.check_weight(W, "bf16", 4, scale=r.scale.cpu().numpy(), codes=r.codes.cpu().numpy(),
+                        deq=bits_of(r.deq), zero_count=int(r.zero_count.item()), ref=ref)

@@ -249,6 +249,30 @@ def test_weight_per_channel(cq, shape, bits):
         parity.check_weight(W, dtype, bits, deq=r.deq.cpu().numpy(), deq_is_f32=True, ref=ref)
 
 
+@pytest.mark.parametrize("shape,group", [((7, 1024), 128), ((3, 8192), 128), ((33, 256), 64), ((5, 512), 256),
+                                         ((9, 96), 32), ((4, 64), 8), ((6, 240), 48), ((5, 100), 10), ((3, 1024), 1024)])
+@pytest.mark.parametrize("bits", [8, 4])
+def test_weight_groupwise(cq, shape, group, bits):
+    R, Cc = shape
+    for dtype in ("bf16", "f16"):
+        W = wl.small_matrix(R, Cc, dtype, 91 + R, scale=0.02, outlier_cols=2, outlier_scale=8.0)
+        W[0, :group] = 0                                     # one all-zero group
+        ref = orc.quantize_weight_groupwise(W, dtype, bits, group)
+        r = cq.quantize_weight_groupwise(to_dev(W, dtype), group, bits)
+        torch.cuda.synchronize()
+        parity.check_weight(W, dtype, bits, scale=r.scale.cpu().numpy(), codes=r.codes.cpu().numpy(),
+                            deq=bits_of(r.deq), zero_count=int(r.zero_count.item()), ref=ref)
+        r = cq.quantize_weight_groupwise(to_dev(W, dtype), group, bits, deq_dtype=torch.float32)
+        parity.check_weight(W, dtype, bits, deq=r.deq.cpu().numpy(), deq_is_f32=True, ref=ref)
+
+
+def test_weight_groupwise_rejects_a_group_that_does_not_divide_the_row(cq):
+    Wd = torch.zeros((4, 100), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(cq.CQError) as e:
+        cq.quantize_weight_groupwise(Wd, 128, 4)
+    assert e.value.status == 2
+
+
 def test_weight_quantizer_equals_alpha_one_activation_path(cq):
     W = wl.small_matrix(64, 1024, "bf16", 61, scale=0.02, outlier_cols=0)
     Wd = to_dev(W, "bf16")

@@ -463,3 +463,23 @@ def test_trend_crossquant_kernel_smaller_than_per_token_on_outlier_data():
     cross = orc.quantize_act(X, cfg.dtype, 0.15, 8).kernel_proportion
     per_token = orc.quantize_act(X, cfg.dtype, 1.0, 8).kernel_proportion
     assert cross < per_token
+
+
+# ------------------------------------------------------------------ group-wise weights
+def test_groupwise_is_per_row_quantization_of_the_reshaped_matrix():
+    """Section 3: reshape to (elements / g) x g, then Eq. 2.  Checked against numpy fp32 ops on the groups."""
+    W = rand_matrix(6, 256, "bf16", 601, scale=0.02, outlier_cols=1, outlier_scale=10.0)
+    w = dec(W, "bf16")
+    for g, bits in [(128, 4), (64, 8), (256, 4)]:
+        r = orc.quantize_weight_groupwise(W, "bf16", bits, g)
+        grp = w.reshape(-1, g)
+        d = (np.abs(grp).max(axis=1) / np.float32(QMAX[bits])).astype(np.float32)[:, None]
+        q = np.rint((grp / d).astype(np.float32)).astype(np.int32)
+        assert np.array_equal(r.codes.reshape(-1, g).astype(np.int32), q)
+        assert np.array_equal(r.scale, d[:, 0])
+        assert r.scale.shape == (6 * 256 // g,)
+    full = orc.quantize_weight_groupwise(W, "bf16", 8, 256)
+    per_channel = orc.quantize_weight_per_channel(W, "bf16", 8)
+    assert np.array_equal(full.codes, per_channel.codes) and np.array_equal(full.scale, per_channel.scale)
+    with pytest.raises(ValueError):
+        orc.quantize_weight_groupwise(W, "bf16", 4, 100)
