@@ -183,6 +183,17 @@ int cq_quantize_weight_groupwise(const void* W, int dtype, int64_t R, int64_t C,
                                  void* codes, float* scale, void* deq, int deq_dtype,
                                  unsigned long long* zero_count, void* stream);
 
+/*
+ * The two indicators of Table 1 (Section 4.2, Cases I and II) from the vectors of one matrix:
+ *   counts[0] = #{(i,j) : c_j >= t_i}                              (Case II)
+ *   counts[1] = #{(i,j) : B~_ij < B_ij}, the CrossQuant zero bound s_ij / 2 (s_ij = fl32(row_scale_i *
+ *               col_scale_j)) against the per-token one, fl32(t_i / qmax) / 2.
+ * t, c, row_scale, col_scale: device vectors as written by cq_quantize_act.  counts: device uint64[2].
+ * Divide by T * I for the proportions the table prints.
+ */
+int cq_case_indicators(const float* t, const float* c, const float* row_scale, const float* col_scale,
+                       int64_t T, int64_t I, int bits, unsigned long long* counts, void* stream);
+
 /* Launch-shape knobs for measurement.  key: "k1_ctas_per_sm", "k3_ctas_per_sm" (resident CTAs per SM
  * the two passes size their grids for; 1..64), "k3_forward" (1: the quantize pass walks the rows in
  * ascending order) or "no_pdl" (1: launch the quantize pass without programmatic dependent launch).  value <= 0 restores the built-in choice.  Results never depend on these.

@@ -343,6 +343,31 @@ void cqo_compare_with_ideal(const uint16_t* X, int dtype, int64_t T, int64_t I, 
     out[2] = far;
 }
 
+/* ---------------------------------------------------------------- Table 1 indicators */
+
+/*
+ * The two indicators of Table 1 (Section 4.2, Cases I / II), over all (i, j) pairs of one matrix:
+ *   out[0] = #{ (i,j) : c_j >= t_i }                                   (Case II)
+ *   out[1] = #{ (i,j) : B~_ij < B_ij } with the zero bounds B~ = s_ij / 2, B = fl32(t_i / qmax) / 2,
+ *            s_ij = fl32(a_i * b_j) the scale the quantizer uses for this alpha.
+ */
+void cqo_case_indicators(const float* t, const float* c, const float* a, const float* b,
+                         int64_t T, int64_t I, int bits, uint64_t* out) {
+    int qmax = qmax_of(bits);
+    uint64_t n_case2 = 0, n_smaller = 0;
+#pragma omp parallel for schedule(static) reduction(+ : n_case2, n_smaller)
+    for (int64_t i = 0; i < T; ++i) {
+        float s_pt = t[i] / (float)qmax;
+        for (int64_t j = 0; j < I; ++j) {
+            float s = a[i] * b[j];
+            if (c[j] >= t[i]) n_case2 += 1;
+            if (0.5f * s < 0.5f * s_pt) n_smaller += 1;
+        }
+    }
+    out[0] = n_case2;
+    out[1] = n_smaller;
+}
+
 int cqo_num_threads(void) {
     int n = 1;
 #ifdef _OPENMP

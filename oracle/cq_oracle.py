@@ -202,3 +202,14 @@ def quantize_weight_groupwise(W: np.ndarray, dtype: str, bits: int, group: int) 
     flat = np.ascontiguousarray(W).reshape(R * Cc // group, group)
     r = quantize_weight_per_channel(flat, dtype, bits)
     return WeightResult(r.scale, r.codes.reshape(R, Cc), r.deq32.reshape(R, Cc), r.deq16.reshape(R, Cc), r.zero_count)
+
+
+def case_indicators(t, c, a, b, bits: int):
+    """(#pairs with c_j >= t_i, #pairs whose CrossQuant zero bound is below the per-token one)."""
+    t = np.ascontiguousarray(t, dtype=np.float32)
+    c = np.ascontiguousarray(c, dtype=np.float32)
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    b = np.ascontiguousarray(b, dtype=np.float32)
+    out = np.zeros(2, dtype=np.uint64)
+    lib().cqo_case_indicators(_p(t), _p(c), _p(a), _p(b), _i64(t.size), _i64(c.size), C.c_int(bits), _p(out))
+    return int(out[0]), int(out[1])

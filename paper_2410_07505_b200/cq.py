@@ -23,7 +23,7 @@ EXPORTS = (
     "cq_workspace_bytes", "cq_quantize_act", "cq_host_scratch_bytes", "cq_quantize_act_host",
     "cq_dequantize", "cq_kernel_count", "cq_kernel_count_x", "cq_quantize_weight_per_channel",
     "cq_set_tuning", "cq_set_timing_events", "cq_quantize_act_noalloc",
-    "cq_quantize_weight_groupwise",
+    "cq_quantize_weight_groupwise", "cq_case_indicators",
 )
 
 
@@ -65,6 +65,7 @@ def lib() -> C.CDLL:
         L.cq_kernel_count_x.argtypes = [vp, ci, i64, i64, i64, dbl, ci, vp, vp, vp, vp, C.c_size_t, vp]
         L.cq_quantize_weight_per_channel.argtypes = [vp, ci, i64, i64, i64, ci, vp, vp, vp, ci, vp, vp]
         L.cq_quantize_weight_groupwise.argtypes = [vp, ci, i64, i64, i64, i64, ci, vp, vp, vp, ci, vp, vp]
+        L.cq_case_indicators.argtypes = [vp, vp, vp, vp, i64, i64, ci, vp, vp]
         L.cq_set_tuning.argtypes = [C.c_char_p, ci]
         L.cq_set_timing_events.argtypes = [vp, vp]
         for name in EXPORTS:
@@ -347,3 +348,12 @@ def quantize_weight_groupwise(W: torch.Tensor, group: int = 128, bits: int = 4, 
                                             _ptr(out.scale), _ptr(out.deq), deq_dt, _ptr(out.zero_count), _stream())
     _check(st, "cq_quantize_weight_groupwise")
     return out
+
+
+def case_indicators(r: ActQuant) -> torch.Tensor:
+    """Table 1 indicators of a quantize_act result: int64[2] on the device,
+    (#pairs with c_j >= t_i, #pairs whose CrossQuant zero bound is below the per-token bound)."""
+    counts = torch.zeros(2, dtype=torch.int64, device=r.t.device)
+    _check(lib().cq_case_indicators(_ptr(r.t), _ptr(r.c), _ptr(r.row_scale), _ptr(r.col_scale), r.t.numel(),
+                                    r.c.numel(), int(r.bits), _ptr(counts), _stream()), "cq_case_indicators")
+    return counts

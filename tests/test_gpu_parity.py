@@ -273,6 +273,20 @@ def test_weight_groupwise_rejects_a_group_that_does_not_divide_the_row(cq):
     assert e.value.status == 2
 
 
+@pytest.mark.parametrize("shape", [(48, 80), (300, 1536), (65, 7), (1, 1)])
+def test_case_indicators(cq, shape):
+    T, I = shape
+    X = wl.small_matrix(T, I, "bf16", 95, dist="laplace", outlier_cols=3, outlier_scale=30.0)
+    if I % 2:
+        X = X[:, :max(1, I)]
+    Xd = to_dev(X, "bf16")
+    for alpha in (0.15, 0.75, 1.0):
+        r = cq.quantize_act(Xd, alpha, 8)
+        got = cq.case_indicators(r).cpu().tolist()
+        ref = orc.quantize_act(X, "bf16", alpha, 8, want_deq32=False, want_deq16=False)
+        assert tuple(got) == orc.case_indicators(ref.t, ref.c, ref.a, ref.b, 8)
+
+
 def test_weight_quantizer_equals_alpha_one_activation_path(cq):
     W = wl.small_matrix(64, 1024, "bf16", 61, scale=0.02, outlier_cols=0)
     Wd = to_dev(W, "bf16")

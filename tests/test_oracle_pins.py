@@ -483,3 +483,27 @@ def test_groupwise_is_per_row_quantization_of_the_reshaped_matrix():
     assert np.array_equal(full.codes, per_channel.codes) and np.array_equal(full.scale, per_channel.scale)
     with pytest.raises(ValueError):
         orc.quantize_weight_groupwise(W, "bf16", 4, 100)
+
+
+# ------------------------------------------------------------------ Table 1 indicators
+def test_case_indicators_brute_force_and_relations():
+    """Cases I / II of Section 4.2: c_j >= t_i  <=>  the CrossQuant bound is not below the per-token
+    bound (alpha < 1, t_i > 0, in real arithmetic); alpha = 1 makes the two bounds equal."""
+    X = rand_matrix(48, 80, "bf16", 701, dist="laplace", outlier_cols=3, outlier_scale=30.0)
+    for alpha in (0.15, 0.45, 0.75):
+        r = orc.quantize_act(X, "bf16", alpha, 8, want_deq32=False, want_deq16=False)
+        n2, nb = orc.case_indicators(r.t, r.c, r.a, r.b, 8)
+        t64, c64 = r.t.astype(np.float64), r.c.astype(np.float64)
+        case2 = c64[None, :] >= t64[:, None]
+        assert n2 == int(case2.sum())
+        # exact evaluation of t^alpha c^(1-alpha) < t; pairs within 1e-6 of equality may go either way
+        ratio = (c64[None, :] / t64[:, None]) ** (1 - alpha)
+        sure = np.abs(ratio - 1) > 1e-6
+        assert int(((ratio < 1) & sure).sum()) <= nb <= int(((ratio < 1) | ~sure).sum())
+        assert abs((n2 + nb) - X.size) <= int((~sure).sum())
+    r1 = orc.quantize_act(X, "bf16", 1.0, 8, want_deq32=False, want_deq16=False)
+    assert orc.case_indicators(r1.t, r1.c, r1.a, r1.b, 8)[1] == 0
+    # hand example: t = (2, 8), c = (4, 8): pairs with c >= t: (0,0), (0,1), (1,1)
+    Xh = wl.to_bits(np.array([[1, 2], [-4, 8]], dtype=np.float32), "f16")
+    rh = orc.quantize_act(Xh, "f16", 0.5, 8)
+    assert orc.case_indicators(rh.t, rh.c, rh.a, rh.b, 8) == (3, 1)
