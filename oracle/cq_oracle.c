@@ -343,6 +343,52 @@ void cqo_compare_with_ideal(const uint16_t* X, int dtype, int64_t T, int64_t I, 
     out[2] = far;
 }
 
+/* ---------------------------------------------------------------- Remove Kernel ---- */
+
+/*
+ * The "Remove Kernel" operator of Figure 1 and Appendix B: the elements of the quantization kernel are
+ * set to zero and every other element is left as it is (not quantized).
+ *   removed  <=>  |u_ij| <= bound_scale / 2,  u_ij = fl32(x_ij / s_ij)  (s_ij == 0 counts as removed);
+ *   bound_scale = 1 removes exactly K(CQ) for this alpha (|u| <= 1/2  <=>  round-half-even(u) == 0);
+ *   other values scale the zero bound B~ and so sweep the removed proportion (Section 4.3).
+ * out16[T*I]: x or +0.  counts[0] = removed, counts[1] = |K(Q)| of per-token quantization (Eq. 1),
+ * counts[2] = |K(CQ)| for this alpha -- all three from one pass over X.
+ */
+int cqo_remove_kernel(const uint16_t* X, int dtype, int64_t T, int64_t I, int64_t ld, double alpha, int bits,
+                      float bound_scale, uint16_t* out16, uint64_t* counts) {
+    if ((bits != 4 && bits != 8) || !(alpha >= 0.0 && alpha <= 1.0) || ld < I || !(bound_scale >= 0.0f)) return -1;
+    int qmax = qmax_of(bits);
+    float* t = (float*)malloc(sizeof(float) * (size_t)(T > 0 ? T : 1));
+    float* c = (float*)malloc(sizeof(float) * (size_t)(I > 0 ? I : 1));
+    float* a = (float*)malloc(sizeof(float) * (size_t)(T > 0 ? T : 1));
+    float* b = (float*)malloc(sizeof(float) * (size_t)(I > 0 ? I : 1));
+    cqo_absmax_rows(X, dtype, T, I, ld, t);
+    cqo_absmax_cols(X, dtype, T, I, ld, c);
+    cqo_scale_vectors(t, c, T, I, alpha, bits, a, b);
+    float half_bound = 0.5f * bound_scale;
+    uint64_t removed = 0, k_pt = 0, k_cq = 0;
+#pragma omp parallel for schedule(static) reduction(+ : removed, k_pt, k_cq)
+    for (int64_t i = 0; i < T; ++i) {
+        float s_pt = t[i] / (float)qmax;
+        for (int64_t j = 0; j < I; ++j) {
+            uint16_t bits16 = X[i * ld + j];
+            float x = decode16(bits16, dtype);
+            float s = a[i] * b[j];
+            float u = (s == 0.0f) ? 0.0f : x / s;
+            int gone = fabsf(u) <= half_bound;
+            if (gone) removed += 1;
+            if (quantize_one(x, s, qmax, 1) == 0) k_cq += 1;
+            if (quantize_one(x, s_pt, qmax, 1) == 0) k_pt += 1;
+            if (out16) out16[i * I + j] = gone ? (uint16_t)0 : bits16;
+        }
+    }
+    counts[0] = removed;
+    counts[1] = k_pt;
+    counts[2] = k_cq;
+    free(t); free(c); free(a); free(b);
+    return 0;
+}
+
 /* ---------------------------------------------------------------- Table 1 indicators */
 
 /*

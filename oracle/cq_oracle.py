@@ -27,7 +27,7 @@ def lib() -> C.CDLL:
         _lib = C.CDLL(path)
         _lib.cqo_kernel_count.restype = C.c_uint64
         _lib.cqo_num_threads.restype = C.c_int
-        for name in ("cqo_quantize_act", "cqo_pack_int4", "cqo_quantize_weight_per_channel"):
+        for name in ("cqo_quantize_act", "cqo_pack_int4", "cqo_quantize_weight_per_channel", "cqo_remove_kernel"):
             getattr(_lib, name).restype = C.c_int
     return _lib
 
@@ -213,3 +213,17 @@ def case_indicators(t, c, a, b, bits: int):
     out = np.zeros(2, dtype=np.uint64)
     lib().cqo_case_indicators(_p(t), _p(c), _p(a), _p(b), _i64(t.size), _i64(c.size), C.c_int(bits), _p(out))
     return int(out[0]), int(out[1])
+
+
+def remove_kernel(X: np.ndarray, dtype: str, alpha: float, bits: int, bound_scale: float = 1.0):
+    """Remove-Kernel operator: (matrix with the kernel elements set to +0 and the rest untouched,
+    #removed, |K(Q)| per-token, |K(CQ)| for alpha)."""
+    ld = _check_bits16(X)
+    T, I = X.shape
+    out = np.empty((T, I), dtype=np.uint16)
+    counts = np.zeros(3, dtype=np.uint64)
+    rc = lib().cqo_remove_kernel(_p(X), DTYPES[dtype], _i64(T), _i64(I), _i64(ld), C.c_double(alpha), C.c_int(bits),
+                                 C.c_float(bound_scale), _p(out), _p(counts))
+    if rc != 0:
+        raise ValueError("cqo_remove_kernel: bad arguments")
+    return out, int(counts[0]), int(counts[1]), int(counts[2])

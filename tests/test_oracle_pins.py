@@ -507,3 +507,40 @@ def test_case_indicators_brute_force_and_relations():
     Xh = wl.to_bits(np.array([[1, 2], [-4, 8]], dtype=np.float32), "f16")
     rh = orc.quantize_act(Xh, "f16", 0.5, 8)
     assert orc.case_indicators(rh.t, rh.c, rh.a, rh.b, 8) == (3, 1)
+
+
+# ------------------------------------------------------------------ Remove Kernel
+def test_remove_kernel_zeroes_exactly_the_kernel_and_touches_nothing_else():
+    X = rand_matrix(96, 160, "f16", 801, outlier_cols=4, outlier_scale=40.0, zero_frac=0.01)
+    x = dec(X, "f16")
+    for alpha in (0.15, 1.0):
+        q = orc.quantize_act(X, "f16", alpha, 8, want_deq32=False, want_deq16=False)
+        out, removed, k_pt, k_cq = orc.remove_kernel(X, "f16", alpha, 8)
+        want = np.where(q.codes == 0, np.uint16(0), X)
+        assert np.array_equal(out, want)
+        assert removed == k_cq == q.zero_count
+        assert k_pt == orc.quantize_act(X, "f16", 1.0, 8, want_deq32=False, want_deq16=False).zero_count
+    # alpha = 1 against numpy fp32 ops: kernel of Eq. 1 is |x / Delta| <= 1/2
+    t = np.abs(x).max(axis=1)
+    u = (x / (t / np.float32(127)).astype(np.float32)[:, None]).astype(np.float32)
+    out, removed, k_pt, _ = orc.remove_kernel(X, "f16", 1.0, 8)
+    assert removed == k_pt == int((np.abs(u) <= 0.5).sum())
+    assert np.array_equal(out, np.where(np.abs(u) <= 0.5, np.uint16(0), X))
+
+
+def test_remove_kernel_bound_scale_sweeps_the_proportion():
+    X = rand_matrix(64, 128, "bf16", 802, outlier_cols=3, outlier_scale=30.0)
+    x = np.abs(dec(X, "bf16"))
+    prev = -1
+    for theta in (0.0, 0.5, 1.0, 2.0, 8.0, 1e9):
+        out, removed, k_pt, k_cq = orc.remove_kernel(X, "bf16", 0.15, 8, theta)
+        assert removed >= prev
+        prev = removed
+        assert int((out == 0).sum()) >= removed            # removed elements are +0; kept ones are bit-identical
+        kept = out != 0
+        assert np.array_equal(out[kept], X[kept])
+        assert k_cq == orc.remove_kernel(X, "bf16", 0.15, 8, 1.0)[1]
+    assert orc.remove_kernel(X, "bf16", 0.15, 8, 0.0)[1] == int((x == 0).sum())
+    assert orc.remove_kernel(X, "bf16", 0.15, 8, 1e9)[1] == X.size
+    with pytest.raises(ValueError):
+        orc.remove_kernel(X, "bf16", 0.15, 8, -1.0)
