@@ -184,6 +184,21 @@ int cq_quantize_weight_groupwise(const void* W, int dtype, int64_t R, int64_t C,
                                  unsigned long long* zero_count, void* stream);
 
 /*
+ * The "Remove Kernel" operator (Figure 1 and Appendix B): the elements of the quantization kernel are set
+ * to zero, every other element is passed through unquantized.  An element is removed when
+ * |fl32(x_ij / s_ij)| <= bound_scale / 2 (s_ij the CrossQuant scale for `alpha`, s_ij == 0 counts as removed).
+ * bound_scale = 1 removes exactly K(CQ) (alpha = 1: the kernel of per-token quantization, Eq. 1); other
+ * values scale the zero bound and so sweep the removed proportion as in Section 4.3.
+ *   out    device [T*I] of X's dtype: x_ij or +0
+ *   counts device uint64[3]: removed elements, |K(Q)| of per-token quantization, |K(CQ)| for `alpha`
+ *          -- the two kernel proportions of Figure 4 from the same pass over X
+ *   workspace as for cq_quantize_act.
+ */
+int cq_remove_kernel(const void* X, int dtype, int64_t T, int64_t I, int64_t ld, double alpha, int bits,
+                     float bound_scale, void* out, unsigned long long* counts,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * The two indicators of Table 1 (Section 4.2, Cases I and II) from the vectors of one matrix:
  *   counts[0] = #{(i,j) : c_j >= t_i}                              (Case II)
  *   counts[1] = #{(i,j) : B~_ij < B_ij}, the CrossQuant zero bound s_ij / 2 (s_ij = fl32(row_scale_i *

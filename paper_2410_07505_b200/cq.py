@@ -23,7 +23,7 @@ EXPORTS = (
     "cq_workspace_bytes", "cq_quantize_act", "cq_host_scratch_bytes", "cq_quantize_act_host",
     "cq_dequantize", "cq_kernel_count", "cq_kernel_count_x", "cq_quantize_weight_per_channel",
     "cq_set_tuning", "cq_set_timing_events", "cq_quantize_act_noalloc",
-    "cq_quantize_weight_groupwise", "cq_case_indicators",
+    "cq_quantize_weight_groupwise", "cq_case_indicators", "cq_remove_kernel",
 )
 
 
@@ -66,6 +66,7 @@ def lib() -> C.CDLL:
         L.cq_quantize_weight_per_channel.argtypes = [vp, ci, i64, i64, i64, ci, vp, vp, vp, ci, vp, vp]
         L.cq_quantize_weight_groupwise.argtypes = [vp, ci, i64, i64, i64, i64, ci, vp, vp, vp, ci, vp, vp]
         L.cq_case_indicators.argtypes = [vp, vp, vp, vp, i64, i64, ci, vp, vp]
+        L.cq_remove_kernel.argtypes = [vp, ci, i64, i64, i64, dbl, ci, C.c_float, vp, vp, vp, C.c_size_t, vp]
         L.cq_set_tuning.argtypes = [C.c_char_p, ci]
         L.cq_set_timing_events.argtypes = [vp, vp]
         for name in EXPORTS:
@@ -357,3 +358,16 @@ def case_indicators(r: ActQuant) -> torch.Tensor:
     _check(lib().cq_case_indicators(_ptr(r.t), _ptr(r.c), _ptr(r.row_scale), _ptr(r.col_scale), r.t.numel(),
                                     r.c.numel(), int(r.bits), _ptr(counts), _stream()), "cq_case_indicators")
     return counts
+
+
+def remove_kernel(X: torch.Tensor, alpha: float = 0.15, bits: int = 8, bound_scale: float = 1.0,
+                  workspace: torch.Tensor | None = None):
+    """Remove-Kernel operator: returns (X with the kernel elements set to +0 and the rest untouched,
+    int64[3] device counts: removed, per-token kernel size, CrossQuant kernel size)."""
+    T, I, ld = _matrix_args(X)
+    ws = workspace if workspace is not None else _workspace(T, I, X.device)
+    out = torch.empty((T, I), dtype=X.dtype, device=X.device)
+    counts = torch.zeros(3, dtype=torch.int64, device=X.device)
+    _check(lib().cq_remove_kernel(_ptr(X), _DT[X.dtype], T, I, ld, float(alpha), int(bits), float(bound_scale), _ptr(out),
+                                  _ptr(counts), _ptr(ws), ws.numel(), _stream()), "cq_remove_kernel")
+    return out, counts

@@ -273,6 +273,21 @@ def test_weight_groupwise_rejects_a_group_that_does_not_divide_the_row(cq):
     assert e.value.status == 2
 
 
+@pytest.mark.parametrize("shape,dtype", [((130, 2056), "bf16"), ((37, 264), "f16"), ((33, 50), "bf16"), ((5, 7), "f16"),
+                                         ((1027, 512), "bf16")])
+def test_remove_kernel(cq, shape, dtype):
+    T, I = shape
+    X = wl.small_matrix(T, I, dtype, 97, outlier_cols=3, outlier_scale=40.0, zero_frac=0.01)
+    X[3 % T, :] = 0
+    Xd = to_dev(X, dtype)
+    for alpha, bits, theta in [(0.15, 8, 1.0), (1.0, 8, 1.0), (0.5, 4, 1.0), (0.15, 8, 0.37), (0.15, 8, 3.0), (0.0, 8, 0.0)]:
+        want, removed, k_pt, k_cq = orc.remove_kernel(X, dtype, alpha, bits, theta)
+        out, counts = cq.remove_kernel(Xd, alpha, bits, theta)
+        torch.cuda.synchronize()
+        assert counts.cpu().tolist() == [removed, k_pt, k_cq]
+        assert np.array_equal(bits_of(out), want)
+
+
 @pytest.mark.parametrize("shape", [(48, 80), (300, 1536), (65, 7), (1, 1)])
 def test_case_indicators(cq, shape):
     T, I = shape
