@@ -708,7 +708,7 @@ int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
     if (bits != 4 && bits != 8) return CQ_ERR_BITS;
     if (!(alpha >= 0.0 && alpha <= 1.0)) return CQ_ERR_ALPHA;
     if (deq != nullptr && deq_dtype != dtype && deq_dtype != CQ_F32) return CQ_ERR_DTYPE;
-    if (bits == 4 && (I % 2) != 0) return CQ_ERR_ALIGN;
+    if (bits == 4 && (I % 2) != 0 && codes != nullptr) return CQ_ERR_ALIGN;      // packed codes need whole bytes
     if (deq != nullptr && !aligned(deq, deq_dtype == CQ_F32 ? 4 : 2)) return CQ_ERR_ALIGN;
     if (zero_count != nullptr && !aligned(zero_count, 8)) return CQ_ERR_ALIGN;
     for (const float* f : {static_cast<const float*>(t), static_cast<const float*>(c),
