@@ -211,8 +211,7 @@ int cq_case_indicators(const float* t, const float* c, const float* row_scale, c
 
 /* Launch-shape knobs for measurement.  key: "k1_ctas_per_sm", "k3_ctas_per_sm" (resident CTAs per SM
  * the two passes size their grids for; 1..64), "k3_forward" (1: the quantize pass walks the rows in
- * ascending order) "no_pdl" (1: launch the quantize pass without programmatic dependent launch) or "no_fuse" (1: always
- * use three launches instead of the single cooperative one).  value <= 0 restores the built-in choice.  Results never depend on these.
+ * ascending order) or "no_pdl" (1: launch the quantize pass without programmatic dependent launch).  value <= 0 restores the built-in choice.  Results never depend on these.
  * Returns CQ_OK or CQ_ERR_SHAPE. */
 int cq_set_tuning(const char* key, int value);
 

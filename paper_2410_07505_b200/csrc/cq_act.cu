@@ -49,21 +49,24 @@ __device__ __forceinline__ void col_scale_of(float cj, double alpha, int qmax, f
 constexpr int kG1 = CQ_K1_GROUP_ROWS; // rows per group of pass 1
 constexpr int kChunkGroups = 32;     // row maxima are flushed to global memory every 32 groups
 
-template <bool ATOMIC, int DT, int G>
-__device__ __forceinline__ void
-absmax_phase(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8, int nstrips,
-             uint16_t* __restrict__ rowpart, uint4* __restrict__ colpart,
-             float* __restrict__ t, float* __restrict__ c) {
-    __shared__ uint16_t s_row[kThreads / 32][kChunkGroups * G];
+template <bool ATOMIC, int DT>
+__global__ void __launch_bounds__(kThreads)
+k1_absmax(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8, int nstrips,
+          uint16_t* __restrict__ rowpart, uint4* __restrict__ colpart,
+          float* __restrict__ t, float* __restrict__ c) {
+    __shared__ uint16_t s_row[kThreads / 32][kChunkGroups * kG1];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int v = blockIdx.x * blockDim.x + tid;
     const bool active = v < I8;
-    const int64_t nfull = T / G;
-    const int64_t ngroups = (T + G - 1) / G;
+    const int64_t nfull = T / kG1;
+    const int64_t ngroups = (T + kG1 - 1) / kG1;
     const int64_t Y = gridDim.y;
     const uint4* xp = X + (active ? v : I8 - 1);
-    const int64_t step = G * Y * ld8;
+    const int64_t step = kG1 * Y * ld8;
     uint4 cm = make_uint4(0, 0, 0, 0);
+    // The quantize pass may be scheduled onto SMs as this grid drains; it waits for this grid to
+    // complete (griddepcontrol.wait) before it touches anything written here.
+    asm volatile("griddepcontrol.launch_dependents;");
 
     auto reduce_row = [&](const uint4& w, int slot) {
         uint4 m = w;
@@ -77,8 +80,8 @@ absmax_phase(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8, int ns
     auto flush_rows = [&](int64_t chunk_g0, int lg) {
         __syncthreads();
         const int nwarps = (blockDim.x + 31) >> 5;
-        for (int k = tid; k < lg * G; k += blockDim.x) {
-            const int64_t row = (chunk_g0 + static_cast<int64_t>(k / G) * Y) * G + (k % G);
+        for (int k = tid; k < lg * kG1; k += blockDim.x) {
+            const int64_t row = (chunk_g0 + static_cast<int64_t>(k / kG1) * Y) * kG1 + (k % kG1);
             if (row < T) {
                 uint32_t m = 0;
                 for (int wdx = 0; wdx < nwarps; ++wdx) m = max(m, static_cast<uint32_t>(s_row[wdx][k]));
@@ -97,28 +100,28 @@ absmax_phase(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8, int ns
     int64_t g = blockIdx.y;
     int64_t chunk_g0 = g;
     int lg = 0;
-    const uint4* p = xp + g * G * ld8;
-    uint4 w[G];
+    const uint4* p = xp + g * kG1 * ld8;
+    uint4 w[kG1];
     if (g < nfull) {
 #pragma unroll
-        for (int u = 0; u < G; ++u) w[u] = ld_nc(p + u * ld8);
+        for (int u = 0; u < kG1; ++u) w[u] = ld_nc(p + u * ld8);
     }
     for (; g < ngroups; g += Y) {
         if (g < nfull) {
             const bool has_next = g + Y < nfull;
             const uint4* pn = p + step;
 #pragma unroll
-            for (int u = 0; u < G; ++u) {
+            for (int u = 0; u < kG1; ++u) {
                 const uint4 cur = w[u];
                 if (has_next) w[u] = ld_nc(pn + u * ld8);
-                reduce_row(cur, lg * G + u);
+                reduce_row(cur, lg * kG1 + u);
             }
             p = pn;
         } else {                                   // the ragged last group: rows past T re-read row T-1
 #pragma unroll
-            for (int u = 0; u < G; ++u) {
-                const int64_t row = min(g * G + u, T - 1);
-                reduce_row(ld_nc(xp + row * ld8), lg * G + u);
+            for (int u = 0; u < kG1; ++u) {
+                const int64_t row = min(g * kG1 + u, T - 1);
+                reduce_row(ld_nc(xp + row * ld8), lg * kG1 + u);
             }
         }
         if (++lg == kChunkGroups) {
@@ -148,17 +151,6 @@ absmax_phase(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8, int ns
             colpart[static_cast<int64_t>(blockIdx.y) * I8 + v] = cm;
         }
     }
-}
-
-template <bool ATOMIC, int DT>
-__global__ void __launch_bounds__(kThreads)
-k1_absmax(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8, int nstrips,
-          uint16_t* __restrict__ rowpart, uint4* __restrict__ colpart,
-          float* __restrict__ t, float* __restrict__ c) {
-    // The next kernel of the stream may be scheduled onto SMs as this grid drains; it waits for this
-    // grid to complete (griddepcontrol.wait) before it touches anything written here.
-    asm volatile("griddepcontrol.launch_dependents;");
-    absmax_phase<ATOMIC, DT, kG1>(X, T, I8, ld8, nstrips, rowpart, colpart, t, c);
 }
 
 // General shapes / alignments: one column per thread, scalar loads, atomic combine (t, c pre-zeroed).
@@ -270,14 +262,13 @@ k2_scales_from_vectors(int64_t T, int64_t I, const float* __restrict__ t_in, con
 // L2) unless `forward` is set; a ragged last group (T not a multiple of 4) is done first by CTA y = 0.
 // Lanes past the last column compute on the last vector and store nothing.
 // DEQ: 0 none, 1 same 16-bit type as X, 2 fp32.
-// COHERENT: the scale vectors were written earlier in the same kernel (fused launch), so they are read
-// past the non-coherent path.
-template <int DT, int BITS, int DEQ, bool CODES, bool COUNT, bool COHERENT>
-__device__ __forceinline__ void
-quantize_phase(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
-               const float* a, const float* ra, const float* b, const float* rb,
-               void* __restrict__ codes, void* __restrict__ deq,
-               unsigned long long* __restrict__ zero_count, int forward) {
+template <int DT, int BITS, int DEQ, bool CODES, bool COUNT>
+__global__ void __launch_bounds__(kThreads, CQ_K3_MIN_CTAS)
+k3_quantize(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
+            const float* __restrict__ a, const float* __restrict__ ra,
+            const float* __restrict__ b, const float* __restrict__ rb,
+            void* __restrict__ codes, void* __restrict__ deq,
+            unsigned long long* __restrict__ zero_count, int forward) {
     const int tid = threadIdx.x, lane = tid & 31;
     const int v = blockIdx.x * blockDim.x + tid;
     const bool active = v < I8;
@@ -287,15 +278,15 @@ quantize_phase(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
     const int64_t Y = gridDim.y;
     unsigned int zeros = 0;
 
-    auto ld_scale4 = [](const float4* q) { return COHERENT ? __ldcg(q) : __ldg(q); };
-    auto ld_scale = [](const float* q) { return COHERENT ? __ldcg(q) : __ldg(q); };
+    // Everything this kernel reads except X is produced by the preceding kernel of the stream.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     if (warp_active) {
         float2 b2[4], rb2[4];
         {
             const float4* bp = reinterpret_cast<const float4*>(b) + static_cast<int64_t>(vv) * 2;
             const float4* rp = reinterpret_cast<const float4*>(rb) + static_cast<int64_t>(vv) * 2;
-            const float4 b0 = ld_scale4(bp), b1 = ld_scale4(bp + 1), q0 = ld_scale4(rp), q1 = ld_scale4(rp + 1);
+            const float4 b0 = __ldg(bp), b1 = __ldg(bp + 1), q0 = __ldg(rp), q1 = __ldg(rp + 1);
             b2[0] = make_float2(b0.x, b0.y); b2[1] = make_float2(b0.z, b0.w);
             b2[2] = make_float2(b1.x, b1.y); b2[3] = make_float2(b1.z, b1.w);
             rb2[0] = make_float2(q0.x, q0.y); rb2[1] = make_float2(q0.z, q0.w);
@@ -344,7 +335,7 @@ quantize_phase(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
         // lanes 0-3 fetch a_i of a group's four rows, lanes 4-7 the reciprocals (rows clamped to T-1)
         auto load_scales = [&](int64_t g) {
             const int64_t row = min((g << 2) + (lane & 3), T - 1);
-            return lane < 8 ? ld_scale((lane < 4 ? a : ra) + row) : 0.0f;
+            return lane < 8 ? __ldg((lane < 4 ? a : ra) + row) : 0.0f;
         };
 
         if ((T & 3) != 0 && blockIdx.y == 0) {          // ragged last group
@@ -387,91 +378,6 @@ quantize_phase(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
         if (!active) zeros = 0;
     }
     if constexpr (COUNT) cta_count_add(zeros, zero_count);
-}
-
-template <int DT, int BITS, int DEQ, bool CODES, bool COUNT>
-__global__ void __launch_bounds__(kThreads, CQ_K3_MIN_CTAS)
-k3_quantize(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
-            const float* __restrict__ a, const float* __restrict__ ra,
-            const float* __restrict__ b, const float* __restrict__ rb,
-            void* __restrict__ codes, void* __restrict__ deq,
-            unsigned long long* __restrict__ zero_count, int forward) {
-    // Everything this kernel reads except X is produced by the preceding kernel of the stream.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    quantize_phase<DT, BITS, DEQ, CODES, COUNT, false>(X, T, I8, ld8, a, ra, b, rb, codes, deq, zero_count, forward);
-}
-
-// ============================================================================ fused launch
-// Both passes and the scale vectors in ONE cooperative launch: the grid is co-resident (the launch
-// fails otherwise), so the CTAs can meet at two grid-wide barriers instead of two kernel boundaries.
-// A barrier is an arrival counter in global memory; waiting is bounded: a CTA that does not see
-// everybody arrive within ~1 s raises the fault word and carries on (results are then garbage but
-// every access stays in bounds), so the kernel always terminates.
-struct FusedArgs {
-    const uint4* X; int64_t T, I; int I8; int64_t ld8; int nstrips;
-    uint16_t* rowpart; uint4* colpart;
-    double alpha; int qmax;
-    float *t, *c, *a, *ra, *b, *rb;
-    void* codes; void* deq; unsigned long long* zero_count;
-    int forward;
-    unsigned int* sync;     // [0] arrival counter (zero at launch), [1] fault word
-};
-
-__device__ __forceinline__ void grid_barrier(unsigned int* counter, unsigned int target, unsigned int* fault) {
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        __threadfence();
-        atomicAdd(counter, 1u);
-        unsigned int seen = 0, polls = 0;
-        for (;;) {
-            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
-            if (seen >= target) break;
-            if (++polls > (1u << 23)) { atomicExch(fault, 1u); break; }
-            __nanosleep(100);
-        }
-        __threadfence();
-    }
-    __syncthreads();
-}
-
-constexpr int kGF = 8;      // rows per group of the absmax phase in the fused launch (2 CTAs per SM)
-
-template <int DT, int BITS, int DEQ, bool CODES, bool COUNT>
-__global__ void __launch_bounds__(kThreads, CQ_K3_MIN_CTAS)
-kf_fused(const FusedArgs p) {
-    const unsigned int nctas = gridDim.x * gridDim.y;
-    absmax_phase<false, DT, kGF>(p.X, p.T, p.I8, p.ld8, p.nstrips, p.rowpart, p.colpart, nullptr, nullptr);
-    grid_barrier(p.sync, nctas, p.sync + 1);
-    {   // finish both reductions, one value per thread: rows first, then columns
-        const int64_t total = static_cast<int64_t>(nctas) * blockDim.x;
-        const int64_t gid = (static_cast<int64_t>(blockIdx.y) * gridDim.x + blockIdx.x) * blockDim.x + threadIdx.x;
-        if (gid == 0 && p.zero_count != nullptr) *p.zero_count = 0ull;
-        const uint16_t* colpart16 = reinterpret_cast<const uint16_t*>(p.colpart);
-        const int64_t cp_ld = static_cast<int64_t>(p.I8) * 8;
-        const int Y = gridDim.y;
-        for (int64_t idx = gid; idx < p.T + p.I; idx += total) {
-            if (idx < p.T) {
-                uint32_t m = 0;
-                for (int sx = 0; sx < p.nstrips; ++sx) m = max(m, static_cast<uint32_t>(__ldcg(p.rowpart + idx * p.nstrips + sx)));
-                const float ti = cvt16<DT>(static_cast<uint16_t>(m));
-                float ai, rai;
-                row_scale_of(ti, p.alpha, p.qmax, ai, rai);
-                p.t[idx] = ti; p.a[idx] = ai; p.ra[idx] = rai;
-            } else {
-                const int64_t j = idx - p.T;
-                uint32_t m = 0;
-#pragma unroll 4
-                for (int y = 0; y < Y; ++y) m = max(m, static_cast<uint32_t>(__ldcg(colpart16 + y * cp_ld + j)));
-                const float cj = cvt16<DT>(static_cast<uint16_t>(m));
-                float bj, rbj;
-                col_scale_of(cj, p.alpha, p.qmax, bj, rbj);
-                p.c[j] = cj; p.b[j] = bj; p.rb[j] = rbj;
-            }
-        }
-    }
-    grid_barrier(p.sync, 2 * nctas, p.sync + 1);
-    quantize_phase<DT, BITS, DEQ, CODES, COUNT, true>(p.X, p.T, p.I8, p.ld8, p.a, p.ra, p.b, p.rb, p.codes, p.deq,
-                                                       p.zero_count, p.forward);
 }
 
 // General shapes / alignments: one thread per pair of adjacent columns.
@@ -630,7 +536,6 @@ static int g_tune_k1_ctas = 0;      // resident CTAs per SM assumed for pass 1 (
 static int g_tune_k3_ctas = 0;      // the same for pass 2
 static int g_tune_k3_forward = 0;   // walk pass 2 in ascending row order
 static int g_tune_no_pdl = 0;       // launch pass 2 without programmatic dependent launch
-static int g_tune_no_fuse = 0;      // never use the single cooperative launch
 static cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
 
 static inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
@@ -668,7 +573,6 @@ Plan make_plan(int64_t T, int64_t I) {
     p.off_b = carve(sizeof(float) * static_cast<size_t>(p.I8) * 8);
     p.off_ra = carve(sizeof(float) * static_cast<size_t>(T));
     p.off_rb = carve(sizeof(float) * static_cast<size_t>(p.I8) * 8);
-    p.off_sync = carve(256);
     p.off_rowpart = carve(sizeof(uint16_t) * static_cast<size_t>(T) * p.nstrips);
     const int64_t ymax = p.ngroups < p.ycap ? (p.ngroups > 0 ? p.ngroups : 1) : p.ycap;
     p.off_colpart = carve(sizeof(uint16_t) * static_cast<size_t>(ymax) * static_cast<size_t>(p.I8) * 8);
@@ -793,55 +697,6 @@ static void launch_k3_deq(const Plan& p, const K3Args& k, int deq_mode, cudaStre
     else launch_k3_flags<DT, BITS, 2>(p, k, st);
 }
 
-// ---- the single cooperative launch (returns CQ_OK, CQ_ERR_CUDA, or -1: not possible here, use three launches)
-static bool cooperative_launch_supported() {
-    int dev = 0, ok = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return false;
-    if (cudaDeviceGetAttribute(&ok, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess) return false;
-    return ok != 0;
-}
-
-template <int DT, int BITS, int DEQ, bool CODES, bool COUNT>
-static int launch_fused_one(const Plan& p, FusedArgs fa, cudaStream_t st) {
-    auto kern = kf_fused<DT, BITS, DEQ, CODES, COUNT>;
-    int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, p.W, 0) != cudaSuccess || per_sm < 1) {
-        cudaGetLastError();
-        return -1;
-    }
-    if (g_tune_k3_ctas > 0 && g_tune_k3_ctas < per_sm) per_sm = g_tune_k3_ctas;
-    int64_t y = static_cast<int64_t>(sm_count()) * per_sm / p.nstrips;
-    if (y > p.ngroups) y = p.ngroups;
-    if (y > p.ycap) y = p.ycap;
-    if (y > 65535) y = 65535;
-    if (y < 1) return -1;                      // more column strips than co-resident CTAs
-    if (cudaMemsetAsync(fa.sync, 0, 2 * sizeof(unsigned int), st) != cudaSuccess) return CQ_ERR_CUDA;
-    void* args[] = {&fa};
-    const cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kern), dim3(p.nstrips, static_cast<unsigned>(y)),
-                                                      dim3(p.W), args, 0, st);
-    if (e != cudaSuccess) {
-        cudaGetLastError();
-        return -1;
-    }
-    return CQ_OK;
-}
-
-template <int DT, int BITS, int DEQ>
-static int launch_fused_flags(const Plan& p, const FusedArgs& fa, cudaStream_t st) {
-    const bool hc = fa.codes != nullptr, hz = fa.zero_count != nullptr;
-    if (hc && hz) return launch_fused_one<DT, BITS, DEQ, true, true>(p, fa, st);
-    if (hc) return launch_fused_one<DT, BITS, DEQ, true, false>(p, fa, st);
-    if (hz) return launch_fused_one<DT, BITS, DEQ, false, true>(p, fa, st);
-    return launch_fused_one<DT, BITS, DEQ, false, false>(p, fa, st);
-}
-
-template <int DT, int BITS>
-static int launch_fused_deq(const Plan& p, const FusedArgs& fa, int deq_mode, cudaStream_t st) {
-    if (deq_mode == 0) return launch_fused_flags<DT, BITS, 0>(p, fa, st);
-    if (deq_mode == 1) return launch_fused_flags<DT, BITS, 1>(p, fa, st);
-    return launch_fused_flags<DT, BITS, 2>(p, fa, st);
-}
-
 // Shared body of cq_quantize_act and cq_kernel_count_x.  t_given/c_given: skip pass 1.
 int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld, double alpha, int bits,
                       const float* t_given, const float* c_given,
@@ -890,28 +745,6 @@ int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
                           T * static_cast<int64_t>(p.I8) < (int64_t(1) << 31);     // 32-bit vector indices
     const unsigned k2v_blocks = static_cast<unsigned>((T + I + kThreads - 1) / kThreads);
 
-    const bool any_out = codes != nullptr || deq != nullptr || zero_count != nullptr;
-    const bool timed = g_ev_before != nullptr && g_ev_after != nullptr;
-
-    // ---- everything in one cooperative launch where that is possible
-    if (!given && fast_in && fast_out && any_out && !timed && !g_tune_no_fuse && cooperative_launch_supported()) {
-        FusedArgs fa{static_cast<const uint4*>(X), T, I, p.I8, ld / 8, p.nstrips, rowpart, reinterpret_cast<uint4*>(colpart),
-                     alpha, qmax, t_dev, c_dev, a_dev, ra_dev, b_dev, rb_dev, codes, deq, zero_count, g_tune_k3_forward,
-                     reinterpret_cast<unsigned int*>(ws + p.off_sync)};
-        const int deq_mode = deq == nullptr ? 0 : (deq_dtype == CQ_F32 ? 2 : 1);
-        int frc;
-        if (dtype == CQ_F16) frc = bits == 8 ? launch_fused_deq<CQ_F16, 8>(p, fa, deq_mode, st) : launch_fused_deq<CQ_F16, 4>(p, fa, deq_mode, st);
-        else frc = bits == 8 ? launch_fused_deq<CQ_BF16, 8>(p, fa, deq_mode, st) : launch_fused_deq<CQ_BF16, 4>(p, fa, deq_mode, st);
-        if (frc == CQ_ERR_CUDA) return frc;
-        if (frc == CQ_OK) {
-            if (c != nullptr && !c_in_place &&
-                cudaMemcpyAsync(c, c_dev, sizeof(float) * I, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return CQ_ERR_CUDA;
-            if (col_scale != nullptr && !b_in_place &&
-                cudaMemcpyAsync(col_scale, b_dev, sizeof(float) * I, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return CQ_ERR_CUDA;
-            return CQ_OK;
-        }
-    }
-
     // ---- pass 1 + scale vectors
     if (given) {
         k2_scales_from_vectors<<<k2v_blocks, kThreads, 0, st>>>(T, I, t_given, c_given, alpha, qmax, a_dev, b_dev,
@@ -940,7 +773,9 @@ int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
     if ((rc = launch_status()) != CQ_OK) return rc;
 
     // ---- pass 2
+    const bool any_out = codes != nullptr || deq != nullptr || zero_count != nullptr;
     if (any_out) {
+        const bool timed = g_ev_before != nullptr && g_ev_after != nullptr;
         if (timed) cudaEventRecord(g_ev_before, st);
         if (fast_in && fast_out) {
             const int deq_mode = deq == nullptr ? 0 : (deq_dtype == CQ_F32 ? 2 : 1);
@@ -1008,7 +843,6 @@ int cq_set_tuning(const char* key, int value) {
     if (eq(key, "k3_ctas_per_sm")) { cq::g_tune_k3_ctas = v; return CQ_OK; }
     if (eq(key, "k3_forward")) { cq::g_tune_k3_forward = v ? 1 : 0; return CQ_OK; }
     if (eq(key, "no_pdl")) { cq::g_tune_no_pdl = v ? 1 : 0; return CQ_OK; }
-    if (eq(key, "no_fuse")) { cq::g_tune_no_fuse = v ? 1 : 0; return CQ_OK; }
     return CQ_ERR_SHAPE;
 }
 

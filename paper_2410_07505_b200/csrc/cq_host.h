@@ -14,7 +14,7 @@ struct Plan {
     int nstrips;   // column strips
     int64_t ngroups;  // groups of 4 rows
     int ycap;      // most CTAs per strip the absmax pass may use (rows of the column-partial buffer)
-    size_t off_t, off_c, off_a, off_b, off_ra, off_rb, off_sync, off_rowpart, off_colpart, total;
+    size_t off_t, off_c, off_a, off_b, off_ra, off_rb, off_rowpart, off_colpart, total;
 };
 
 Plan make_plan(int64_t T, int64_t I);

@@ -162,20 +162,14 @@ def test_tiling_knobs_do_not_change_results(cq):
             cq.set_tuning(key, 0)
 
 
-@pytest.mark.parametrize("knob", ["no_fuse", "no_pdl"])
-def test_three_launch_path_gives_the_same_results(cq, knob):
-    """The single cooperative launch is the default; the three-launch path (and its variant without
-    programmatic dependent launch) must agree with the oracle just the same."""
+def test_launch_without_programmatic_dependent_launch_gives_the_same_results(cq):
     try:
-        cq.set_tuning("no_fuse", 1)
-        cq.set_tuning(knob, 1)
-        for (T, I), dtype in [((130, 2056), "bf16"), ((257, 776), "f16"), ((3, 16), "bf16"), ((1027, 4104), "f16")]:
+        cq.set_tuning("no_pdl", 1)
+        for (T, I), dtype in [((130, 2056), "bf16"), ((257, 776), "f16"), ((1027, 4104), "f16")]:
             X = wl.small_matrix(T, I, dtype, 3000 + T, outlier_cols=2, zero_frac=0.01)
-            for bits, alpha in [(8, 0.15), (4, 0.5), (8, 1.0)]:
+            for bits, alpha in [(8, 0.15), (4, 0.5)]:
                 run_and_check(cq, X, dtype, alpha, bits)
-            run_and_check(cq, X, dtype, 0.15, 8, deq_f32=True)
     finally:
-        cq.set_tuning("no_fuse", 0)
         cq.set_tuning("no_pdl", 0)
 
 
