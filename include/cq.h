@@ -211,9 +211,15 @@ int cq_case_indicators(const float* t, const float* c, const float* row_scale, c
 
 /* Launch-shape knobs for measurement.  key: "k1_ctas_per_sm", "k3_ctas_per_sm" (resident CTAs per SM
  * the two passes size their grids for; 1..64), "k3_forward" (1: the quantize pass walks the rows in
- * ascending order) or "no_pdl" (1: launch the quantize pass without programmatic dependent launch).  value <= 0 restores the built-in choice.  Results never depend on these.
+ * ascending order) or "no_pdl" (1: launch the quantize pass without programmatic dependent launch), "no_stage" (1: the quantize pass
+ * loads rows straight into registers instead of staging them in shared memory with bulk copies).  value <= 0 restores the built-in choice.  Results never depend on these.
  * Returns CQ_OK or CQ_ERR_SHAPE. */
 int cq_set_tuning(const char* key, int value);
+
+/* Health check.  The quantize pass waits for its asynchronous row copies with a bounded number of polls;
+ * if a wait ever gives up, a device flag is raised (results of that call are then undefined).  This
+ * copies the flag of the current device to *fault_host (0 = never happened).  Synchronises the device. */
+int cq_stage_fault(unsigned int* fault_host);
 
 /* Measurement hook: while both are non-NULL, cq_quantize_act records the two cudaEvent_t (passed
  * as void*, owned by the caller) on its stream immediately before and after the quantize pass, so

@@ -23,7 +23,7 @@ EXPORTS = (
     "cq_workspace_bytes", "cq_quantize_act", "cq_host_scratch_bytes", "cq_quantize_act_host",
     "cq_dequantize", "cq_kernel_count", "cq_kernel_count_x", "cq_quantize_weight_per_channel",
     "cq_set_tuning", "cq_set_timing_events", "cq_quantize_act_noalloc",
-    "cq_quantize_weight_groupwise", "cq_case_indicators", "cq_remove_kernel",
+    "cq_quantize_weight_groupwise", "cq_case_indicators", "cq_remove_kernel", "cq_stage_fault",
 )
 
 
@@ -67,6 +67,7 @@ def lib() -> C.CDLL:
         L.cq_quantize_weight_groupwise.argtypes = [vp, ci, i64, i64, i64, i64, ci, vp, vp, vp, ci, vp, vp]
         L.cq_case_indicators.argtypes = [vp, vp, vp, vp, i64, i64, ci, vp, vp]
         L.cq_remove_kernel.argtypes = [vp, ci, i64, i64, i64, dbl, ci, C.c_float, vp, vp, vp, C.c_size_t, vp]
+        L.cq_stage_fault.argtypes = [vp]
         L.cq_set_tuning.argtypes = [C.c_char_p, ci]
         L.cq_set_timing_events.argtypes = [vp, vp]
         for name in EXPORTS:
@@ -371,3 +372,10 @@ def remove_kernel(X: torch.Tensor, alpha: float = 0.15, bits: int = 8, bound_sca
     _check(lib().cq_remove_kernel(_ptr(X), _DT[X.dtype], T, I, ld, float(alpha), int(bits), float(bound_scale), _ptr(out),
                                   _ptr(counts), _ptr(ws), ws.numel(), _stream()), "cq_remove_kernel")
     return out, counts
+
+
+def stage_fault() -> int:
+    """1 if a bounded wait on a staged row copy ever gave up on the current device, else 0."""
+    flag = C.c_uint(0)
+    _check(lib().cq_stage_fault(C.byref(flag)), "cq_stage_fault")
+    return int(flag.value)

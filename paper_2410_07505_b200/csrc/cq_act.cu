@@ -262,13 +262,21 @@ k2_scales_from_vectors(int64_t T, int64_t I, const float* __restrict__ t_in, con
 // L2) unless `forward` is set; a ragged last group (T not a multiple of 4) is done first by CTA y = 0.
 // Lanes past the last column compute on the last vector and store nothing.
 // DEQ: 0 none, 1 same 16-bit type as X, 2 fp32.
-template <int DT, int BITS, int DEQ, bool CODES, bool COUNT>
+// STAGED: the rows are brought into a ring of shared-memory stages by asynchronous bulk copies
+// (kStages groups of four rows per CTA, issued by thread 0 one group ahead of the ring's free slot), so
+// the bytes in flight per SM are set by the ring (up to 3 x 16 KB per CTA) instead of by registers.
+constexpr int kStages = 4;
+__device__ unsigned int g_stage_fault = 0;      // set if a bounded wait on a stage ever gave up
+
+template <int DT, int BITS, int DEQ, bool CODES, bool COUNT, bool STAGED>
 __global__ void __launch_bounds__(kThreads, CQ_K3_MIN_CTAS)
 k3_quantize(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
             const float* __restrict__ a, const float* __restrict__ ra,
             const float* __restrict__ b, const float* __restrict__ rb,
             void* __restrict__ codes, void* __restrict__ deq,
             unsigned long long* __restrict__ zero_count, int forward) {
+    extern __shared__ __align__(128) unsigned char s_dyn[];
+    __shared__ uint64_t s_full[kStages];
     const int tid = threadIdx.x, lane = tid & 31;
     const int v = blockIdx.x * blockDim.x + tid;
     const bool active = v < I8;
@@ -281,7 +289,7 @@ k3_quantize(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
     // Everything this kernel reads except X is produced by the preceding kernel of the stream.
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    if (warp_active) {
+    if (warp_active || STAGED) {
         float2 b2[4], rb2[4];
         {
             const float4* bp = reinterpret_cast<const float4*>(b) + static_cast<int64_t>(vv) * 2;
@@ -338,7 +346,7 @@ k3_quantize(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
             return lane < 8 ? __ldg((lane < 4 ? a : ra) + row) : 0.0f;
         };
 
-        if ((T & 3) != 0 && blockIdx.y == 0) {          // ragged last group
+        if ((T & 3) != 0 && blockIdx.y == 0 && warp_active) {          // ragged last group
             const float arv = load_scales(nfull);
             for (int u = 0; u < static_cast<int>(T & 3); ++u) {
                 const int64_t row = (nfull << 2) + u;
@@ -348,8 +356,52 @@ k3_quantize(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
             }
         }
 
+        if constexpr (STAGED) {
+            uint4* stage = reinterpret_cast<uint4*>(s_dyn);               // [kStages][4 rows][blockDim.x]
+            const int Wv = blockDim.x;
+            const int strip0 = blockIdx.x * Wv;
+            const uint32_t seg_bytes = static_cast<uint32_t>(min(Wv, I8 - strip0)) * 16u;
+            const int64_t first = blockIdx.y;
+            const int64_t mine = first < nfull ? (nfull - first + Y - 1) / Y : 0;      // groups of this CTA
+            auto group_at = [&](int64_t k) { const int64_t pos = first + k * Y; return forward ? pos : nfull - 1 - pos; };
+            auto issue = [&](int64_t k) {                                 // thread 0 only
+                if (k >= mine) return;
+                const int st = static_cast<int>(k % kStages);
+                const uint4* src = X + (group_at(k) << 2) * ld8 + strip0;
+                mbar_expect_tx(&s_full[st], 4u * seg_bytes);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) bulk_load(stage + (st * 4 + u) * Wv, src + u * ld8, seg_bytes, &s_full[st]);
+            };
+            if (tid == 0) {
+#pragma unroll
+                for (int st = 0; st < kStages; ++st) mbar_init(&s_full[st], 1);
+                mbar_init_fence();
+            }
+            __syncthreads();
+            if (tid == 0) {
+                for (int k = 0; k < kStages - 1; ++k) issue(k);
+            }
+            for (int64_t k = 0; k < mine; ++k) {
+                const int64_t g = group_at(k);
+                const float arv = load_scales(g);
+                __syncthreads();                                          // everybody is done with group k-1: its stage is free
+                if (tid == 0) issue(k + kStages - 1);
+                const int st = static_cast<int>(k % kStages);
+                if (!mbar_wait(&s_full[st], static_cast<uint32_t>((k / kStages) & 1))) atomicExch(&g_stage_fault, 1u);
+                if (warp_active) {
+                    const int vec = static_cast<int>((g << 2) * I8 + vv);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        uint4 cur = stage[(st * 4 + u) * Wv + tid];
+                        do_row(cur, nullptr, false, __shfl_sync(0xFFFFFFFFu, arv, u), __shfl_sync(0xFFFFFFFFu, arv, 4 + u),
+                               vec + u * I8);
+                    }
+                }
+            }
+        }
+
         int64_t pos = blockIdx.y;
-        if (pos < nfull) {
+        if (!STAGED && pos < nfull) {
             const int64_t dgroups = forward ? Y : -Y;
             int64_t g = forward ? pos : nfull - 1 - pos;
             const int64_t xstep = 4 * dgroups * ld8;
@@ -536,6 +588,7 @@ static int g_tune_k1_ctas = 0;      // resident CTAs per SM assumed for pass 1 (
 static int g_tune_k3_ctas = 0;      // the same for pass 2
 static int g_tune_k3_forward = 0;   // walk pass 2 in ascending row order
 static int g_tune_no_pdl = 0;       // launch pass 2 without programmatic dependent launch
+static int g_tune_no_stage = 0;     // pass 2 loads rows straight into registers instead of staging them
 static cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
 
 static inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
@@ -653,14 +706,14 @@ static int absmax_atomic(const void* X, int dtype, int64_t T, int64_t I, int64_t
 // Programmatic dependent launch: the kernel's CTAs may become resident while the previous kernel of
 // the stream drains; the kernel itself waits (griddepcontrol.wait) before reading what that one wrote.
 template <typename... KArgs, typename... Args>
-static void launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+static void launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = g_tune_no_pdl ? 0 : 1;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = grid;
     cfg.blockDim = block;
-    cfg.dynamicSmemBytes = 0;
+    cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
@@ -675,9 +728,26 @@ struct K3Args {
 
 template <int DT, int BITS, int DEQ, bool CODES, bool COUNT>
 static void launch_k3_one(const Plan& p, const K3Args& k, cudaStream_t st) {
-    auto kern = k3_quantize<DT, BITS, DEQ, CODES, COUNT>;
+    if (!g_tune_no_stage) {
+        auto kern = k3_quantize<DT, BITS, DEQ, CODES, COUNT, true>;
+        const size_t smem = static_cast<size_t>(kStages) * 4 * p.W * 16;
+        int per_sm = 0;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) == cudaSuccess &&
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, p.W, smem) == cudaSuccess && per_sm >= 1) {
+            if (g_tune_k3_ctas > 0) per_sm = g_tune_k3_ctas;
+            int64_t y = static_cast<int64_t>(sm_count()) * per_sm / p.nstrips;
+            if (y > p.ngroups) y = p.ngroups;
+            if (y > 65535) y = 65535;
+            if (y < 1) y = 1;
+            launch_dependent(kern, dim3(p.nstrips, static_cast<unsigned>(y)), dim3(p.W), smem, st, k.X, k.T, k.I8, k.ld8, k.a,
+                             k.ra, k.b, k.rb, k.codes, k.deq, k.zc, g_tune_k3_forward);
+            return;
+        }
+        cudaGetLastError();
+    }
+    auto kern = k3_quantize<DT, BITS, DEQ, CODES, COUNT, false>;
     const int Y = resident_y(kern, p.W, p.nstrips, p.ngroups, g_tune_k3_ctas, 0);
-    launch_dependent(kern, dim3(p.nstrips, Y), dim3(p.W), st, k.X, k.T, k.I8, k.ld8, k.a, k.ra, k.b, k.rb, k.codes,
+    launch_dependent(kern, dim3(p.nstrips, Y), dim3(p.W), 0, st, k.X, k.T, k.I8, k.ld8, k.a, k.ra, k.b, k.rb, k.codes,
                      k.deq, k.zc, g_tune_k3_forward);
 }
 
@@ -755,12 +825,12 @@ int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
         const uint4* cp4 = reinterpret_cast<const uint4*>(colpart);
         if (dtype == CQ_F16) {
             const int Y = launch_k1<false, CQ_F16>(p, X, T, ld, rowpart, colpart, nullptr, nullptr, st);
-            launch_dependent(k2_scales_from_partials<CQ_F16>, dim3(blocks), dim3(kThreads), st, T, I, p.I8, p.nstrips, Y,
+            launch_dependent(k2_scales_from_partials<CQ_F16>, dim3(blocks), dim3(kThreads), 0, st, T, I, p.I8, p.nstrips, Y,
                              col_ctas, static_cast<const uint16_t*>(rowpart), cp4, alpha, qmax, t_dev, c_dev, a_dev, b_dev,
                              ra_dev, rb_dev, zero_count);
         } else {
             const int Y = launch_k1<false, CQ_BF16>(p, X, T, ld, rowpart, colpart, nullptr, nullptr, st);
-            launch_dependent(k2_scales_from_partials<CQ_BF16>, dim3(blocks), dim3(kThreads), st, T, I, p.I8, p.nstrips, Y,
+            launch_dependent(k2_scales_from_partials<CQ_BF16>, dim3(blocks), dim3(kThreads), 0, st, T, I, p.I8, p.nstrips, Y,
                              col_ctas, static_cast<const uint16_t*>(rowpart), cp4, alpha, qmax, t_dev, c_dev, a_dev, b_dev,
                              ra_dev, rb_dev, zero_count);
         }
@@ -843,7 +913,13 @@ int cq_set_tuning(const char* key, int value) {
     if (eq(key, "k3_ctas_per_sm")) { cq::g_tune_k3_ctas = v; return CQ_OK; }
     if (eq(key, "k3_forward")) { cq::g_tune_k3_forward = v ? 1 : 0; return CQ_OK; }
     if (eq(key, "no_pdl")) { cq::g_tune_no_pdl = v ? 1 : 0; return CQ_OK; }
+    if (eq(key, "no_stage")) { cq::g_tune_no_stage = v ? 1 : 0; return CQ_OK; }
     return CQ_ERR_SHAPE;
+}
+
+int cq_stage_fault(unsigned int* fault_host) {
+    if (fault_host == nullptr) return CQ_ERR_NULL;
+    return cudaMemcpyFromSymbol(fault_host, cq::g_stage_fault, sizeof(unsigned int)) == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
 }
 
 int cq_set_timing_events(void* before_quantize_pass, void* after_quantize_pass) {
