@@ -15,6 +15,9 @@
 #ifndef CQ_K3_MIN_CTAS
 #define CQ_K3_MIN_CTAS 2
 #endif
+#ifndef CQ_STAGES
+#define CQ_STAGES 4
+#endif
 
 namespace cq {
 
@@ -265,16 +268,19 @@ k2_scales_from_vectors(int64_t T, int64_t I, const float* __restrict__ t_in, con
 // STAGED: the rows are brought into a ring of shared-memory stages by asynchronous bulk copies
 // (kStages groups of four rows per CTA, issued by thread 0 one group ahead of the ring's free slot), so
 // the bytes in flight per SM are set by the ring (up to 3 x 16 KB per CTA) instead of by registers.
-constexpr int kStages = 4;
+constexpr int kStages = CQ_STAGES;
 __device__ unsigned int g_stage_fault = 0;      // set if a bounded wait on a stage ever gave up
 
-template <int DT, int BITS, int DEQ, bool CODES, bool COUNT, bool STAGED>
-__global__ void __launch_bounds__(kThreads, CQ_K3_MIN_CTAS)
+// MODE 0: rows straight into registers; MODE 2 / 3: staged, compiled for 2 / 3 resident CTAs per SM
+// (two are faster when X streams from HBM, three when it is served by L2).
+template <int DT, int BITS, int DEQ, bool CODES, bool COUNT, int MODE>
+__global__ void __launch_bounds__(kThreads, MODE == 0 ? CQ_K3_MIN_CTAS : MODE)
 k3_quantize(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
             const float* __restrict__ a, const float* __restrict__ ra,
             const float* __restrict__ b, const float* __restrict__ rb,
             void* __restrict__ codes, void* __restrict__ deq,
             unsigned long long* __restrict__ zero_count, int forward) {
+    constexpr bool STAGED = MODE != 0;
     extern __shared__ __align__(128) unsigned char s_dyn[];
     __shared__ uint64_t s_full[kStages];
     const int tid = threadIdx.x, lane = tid & 31;
@@ -726,26 +732,37 @@ struct K3Args {
     void* codes; void* deq; unsigned long long* zc;
 };
 
+template <int DT, int BITS, int DEQ, bool CODES, bool COUNT, int MODE>
+static bool launch_k3_staged(const Plan& p, const K3Args& k, cudaStream_t st) {
+    auto kern = k3_quantize<DT, BITS, DEQ, CODES, COUNT, MODE>;
+    const size_t smem = static_cast<size_t>(kStages) * 4 * p.W * 16;
+    int per_sm = 0;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, p.W, smem) != cudaSuccess || per_sm < 1) {
+        cudaGetLastError();
+        return false;
+    }
+    int64_t y = static_cast<int64_t>(sm_count()) * per_sm / p.nstrips;
+    if (y > p.ngroups) y = p.ngroups;
+    if (y > 65535) y = 65535;
+    if (y < 1) y = 1;
+    launch_dependent(kern, dim3(p.nstrips, static_cast<unsigned>(y)), dim3(p.W), smem, st, k.X, k.T, k.I8, k.ld8, k.a, k.ra,
+                     k.b, k.rb, k.codes, k.deq, k.zc, g_tune_k3_forward);
+    return true;
+}
+
 template <int DT, int BITS, int DEQ, bool CODES, bool COUNT>
 static void launch_k3_one(const Plan& p, const K3Args& k, cudaStream_t st) {
     if (!g_tune_no_stage) {
-        auto kern = k3_quantize<DT, BITS, DEQ, CODES, COUNT, true>;
-        const size_t smem = static_cast<size_t>(kStages) * 4 * p.W * 16;
-        int per_sm = 0;
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) == cudaSuccess &&
-            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, p.W, smem) == cudaSuccess && per_sm >= 1) {
-            if (g_tune_k3_ctas > 0) per_sm = g_tune_k3_ctas;
-            int64_t y = static_cast<int64_t>(sm_count()) * per_sm / p.nstrips;
-            if (y > p.ngroups) y = p.ngroups;
-            if (y > 65535) y = 65535;
-            if (y < 1) y = 1;
-            launch_dependent(kern, dim3(p.nstrips, static_cast<unsigned>(y)), dim3(p.W), smem, st, k.X, k.T, k.I8, k.ld8, k.a,
-                             k.ra, k.b, k.rb, k.codes, k.deq, k.zc, g_tune_k3_forward);
-            return;
-        }
-        cudaGetLastError();
+        // matrices that stream from HBM run two CTAs per SM, those L2 can hold run three
+        const int64_t bytes = k.T * k.ld8 * 16;
+        int mode = bytes > (int64_t(120) << 20) ? 2 : 3;
+        if (g_tune_k3_ctas == 2 || g_tune_k3_ctas == 3) mode = g_tune_k3_ctas;
+        const bool ok = mode == 2 ? launch_k3_staged<DT, BITS, DEQ, CODES, COUNT, 2>(p, k, st)
+                                  : launch_k3_staged<DT, BITS, DEQ, CODES, COUNT, 3>(p, k, st);
+        if (ok) return;
     }
-    auto kern = k3_quantize<DT, BITS, DEQ, CODES, COUNT, false>;
+    auto kern = k3_quantize<DT, BITS, DEQ, CODES, COUNT, 0>;
     const int Y = resident_y(kern, p.W, p.nstrips, p.ngroups, g_tune_k3_ctas, 0);
     launch_dependent(kern, dim3(p.nstrips, Y), dim3(p.W), 0, st, k.X, k.T, k.I8, k.ld8, k.a, k.ra, k.b, k.rb, k.codes,
                      k.deq, k.zc, g_tune_k3_forward);
