@@ -42,8 +42,8 @@ HOOK_EVERY = 8
 
 # DRAM traffic of the quantize pass from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum
 # per launch), valid only for the kernel sources whose digest is recorded with it.
-NCU_TRAFFIC = {"sources_sha256": "0f231ec4fff1c168e931e6345b77cc9484e05f61b23225b346cf92a21f860c20",
-               "bytes_per_launch": 532098048}   # 235,176,192 read + 296,921,856 written
+NCU_TRAFFIC = {"sources_sha256": "c355f682e4bf8899c8428f2ffe46ec6eb0ed8ab7fbad0d654be766130158b5d1",
+               "bytes_per_launch": 528244480}   # 235,183,616 read + 293,060,864 written
 
 
 def kernel_sources_digest() -> str:
