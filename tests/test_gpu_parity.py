@@ -237,7 +237,8 @@ def test_kernel_count_straight_from_x(cq, bits):
         assert int(cq.kernel_count_x(Xd, alpha, bits, t, c).item()) == ref.zero_count
 
 
-WEIGHT_SHAPES = [(1, 8), (5, 264), (40, 2056), (7, 8192), (3, 28672), (33, 50), (6, 1001), (2, 110600)]
+WEIGHT_SHAPES = [(1, 8), (5, 264), (40, 2056), (7, 8192), (3, 28672), (33, 50), (6, 1001), (2, 110600), (5, 12296),
+                 (3, 57352), (2, 300000)]
 
 
 @pytest.mark.parametrize("shape", WEIGHT_SHAPES)
