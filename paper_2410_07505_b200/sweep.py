@@ -63,6 +63,27 @@ def time_weight(Wd: torch.Tensor, bits: int, flush, iters: int) -> dict:
             "kernel_proportion": int(out.zero_count.item()) / n}
 
 
+def time_extra_ops(Xd: torch.Tensor, alpha: float, flush, iters: int) -> dict:
+    """Remove-Kernel operator, Table 1 indicators and the count-only pass on one activation matrix."""
+    T, I = Xd.shape
+    n = T * I
+    ws = torch.empty(cq.workspace_bytes(T, I), dtype=torch.uint8, device=Xd.device)
+    r = cq.quantize_act(Xd, alpha, 8)
+    t, c = cq.absmax_rows_cols(Xd)
+    us_rm = _time(lambda: cq.remove_kernel(Xd, alpha, 8, 1.0, ws), flush, iters)
+    us_ind = _time(lambda: cq.case_indicators(r), flush, iters)
+    us_cnt = _time(lambda: cq.kernel_count_x(Xd, alpha, 8, t, c, ws), flush, iters)
+    us_abs = _time(lambda: cq.absmax_rows_cols(Xd), flush, iters)
+    _, counts = cq.remove_kernel(Xd, alpha, 8, 1.0, ws)
+    ind = cq.case_indicators(r).cpu().tolist()
+    cnt = counts.cpu().tolist()
+    return {"remove_kernel_us": round(us_rm, 1), "remove_kernel_gbs": round(6 * n / us_rm / 1e3, 1),
+            "case_indicators_us": round(us_ind, 1), "kernel_count_x_us": round(us_cnt, 1),
+            "absmax_rows_cols_us": round(us_abs, 1), "absmax_gbs": round(2 * n / us_abs / 1e3, 1),
+            "kernel_proportion_per_token": cnt[1] / n, "kernel_proportion_crossquant": cnt[2] / n,
+            "share_c_ge_t": ind[0] / n, "share_bound_smaller": ind[1] / n}
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--iters", type=int, default=30)
@@ -79,6 +100,10 @@ def main() -> None:
                 row = {"config": name, "shape": [cfg.T, cfg.I], "dtype": cfg.dtype, "bits": bits, "alpha": alpha}
                 row.update(time_activation(Xd, bits, alpha, flush, args.iters))
                 print(json.dumps(row), flush=True)
+        if name != "tiny":
+            row = {"config": name, "shape": [cfg.T, cfg.I], "dtype": cfg.dtype, "ops": "diagnostics", "alpha": args.alpha}
+            row.update(time_extra_ops(Xd, args.alpha, flush, args.iters))
+            print(json.dumps(row), flush=True)
         del Xd
     for k, shape in enumerate(wl.SWEEP_WEIGHT_SHAPES):
         Wd = _dev(wl.sweep_weight(0, k), "bf16")
@@ -86,7 +111,12 @@ def main() -> None:
             row = {"config": f"weight_{shape[0]}x{shape[1]}", "shape": list(shape), "dtype": "bf16", "bits": bits}
             row.update(time_weight(Wd, bits, flush, args.iters))
             print(json.dumps(row), flush=True)
-        del Wd
+        out = cq.quantize_weight_groupwise(Wd, 128, 4)
+        us = _time(lambda: cq.quantize_weight_groupwise(Wd, 128, 4, out=out), flush, args.iters)
+        print(json.dumps({"config": f"weight_{shape[0]}x{shape[1]}_g128", "shape": list(shape), "dtype": "bf16", "bits": 4,
+                          "us_l2_flushed": round(us, 1), "gbs": round(4.5 * Wd.numel() / us / 1e3, 1),
+                          "kernel_proportion": int(out.zero_count.item()) / Wd.numel()}), flush=True)
+        del Wd, out
 
     total_us = 0.0
     for layer in range(args.layers):
