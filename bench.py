@@ -249,11 +249,13 @@ def main() -> None:
     value = whole_job_gbs(n, K, world, total_ms)
     zero_count = int(buf.zero_count.item())
 
-    # ---- end to end: host buffers in, host buffers out, through cq_quantize_act_host
+    # ---- end to end: host buffers in, host buffers out, through cq_quantize_act_host.
+    # (a) one call after the other on one stream; (b) the same calls issued alternately on two streams with
+    # their own buffers, so one step's download overlaps the next step's upload (PCIe is full duplex).
     Xp = Xh.pin_memory()
-    hb = cq.HostBuffers(T, I, torch.bfloat16, BITS)
+    hbs = [cq.HostBuffers(T, I, torch.bfloat16, BITS) for _ in range(2)]
     Ke = max(1, args.e2e_steps)
-    for _ in range(2):
+    for hb in hbs:
         cq.quantize_act_host(Xp, ALPHA, BITS, buffers=hb)
     torch.cuda.synchronize()
     e0 = [torch.cuda.Event(enable_timing=True) for _ in range(Ke)]
@@ -262,12 +264,57 @@ def main() -> None:
         dist.barrier()
     for k in range(Ke):
         e0[k].record()
-        cq.quantize_act_host(Xp, ALPHA, BITS, buffers=hb)
+        cq.quantize_act_host(Xp, ALPHA, BITS, buffers=hbs[0])
         e1[k].record()
     torch.cuda.synchronize()
-    e2e_ms = max_over_ranks(sum(a.elapsed_time(b) for a, b in zip(e0, e1)), "cuda")
+    serial_ms = max_over_ranks(sum(a.elapsed_time(b) for a, b in zip(e0, e1)), "cuda")
+    e2e_serial = whole_job_gbs(n, Ke, world, serial_ms)
+    assert int(hbs[0].zero_count.item()) == zero_count
+
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    p0.record()
+    for st in streams:
+        st.wait_event(p0)
+    for k in range(Ke):
+        with torch.cuda.stream(streams[k % 2]):
+            cq.quantize_act_host(Xp, ALPHA, BITS, buffers=hbs[k % 2])
+    for st in streams:
+        torch.cuda.current_stream().wait_stream(st)
+    p1.record()
+    torch.cuda.synchronize()
+    e2e_ms = max_over_ranks(p0.elapsed_time(p1), "cuda")
     e2e_value = whole_job_gbs(n, Ke, world, e2e_ms)
-    assert int(hb.zero_count.item()) == zero_count
+    assert int(hbs[1 if Ke > 1 else 0].zero_count.item()) == zero_count
+    hb = hbs[0]
+
+    # ---- also: INT4 codes on the same matrix and the per-channel weight quantizer (not part of `value`)
+    def timed(fn, iters=40):
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
+        for _ in range(3):
+            fn()
+        for a_, b_ in evs:
+            flush.zero_()
+            a_.record()
+            fn()
+            b_.record()
+        torch.cuda.synchronize()
+        return statistics.median(a_.elapsed_time(b_) for a_, b_ in evs)
+    also = {}
+    if rank == 0:
+        buf4 = cq.ActBuffers(T, I, torch.bfloat16, 4)
+        ms4 = timed(lambda: cq.quantize_act(Xd, ALPHA, 4, buffers=buf4))
+        also["act_int4"] = {"ms_per_step": ms4, "gbs": 6.5 * n / (ms4 * 1e-3) / 1e9, "bytes_per_element": 6.5}
+        del buf4
+        Wd = torch.from_numpy(wl.sweep_weight(0, 2).view(np.int16)).view(torch.bfloat16).cuda()
+        wout = cq.quantize_weight_per_channel(Wd, 8)
+        msw = timed(lambda: cq.quantize_weight_per_channel(Wd, 8, out=wout))
+        also["weight_per_channel_int8_28672x8192"] = {"ms": msw, "gbs": 5.0 * Wd.numel() / (msw * 1e-3) / 1e9,
+                                                       "bytes_per_element": 5.0}
+        del Wd, wout
 
     if rank != 0:
         if world > 1:
@@ -295,7 +342,10 @@ def main() -> None:
         "gpu_launches": 3 * K,
         "e2e": {"value": e2e_value, "unit": UNIT, "steps": Ke,
                 "h2d_bytes_per_step": X.nbytes, "d2h_bytes_per_step": hb.d2h_bytes(),
-                "api": "cq_quantize_act_host (pinned host buffers; copies inside the timed region)"},
+                "api": "cq_quantize_act_host (pinned host buffers; copies inside the timed region), calls issued "
+                       "alternately on two streams so a step's download overlaps the next step's upload",
+                "one_stream_value": e2e_serial},
+        "also": also,
         "roofline": {"bound": "hbm", "kernel": "k3_quantize (quantize / pack / dequantize / zero-count pass)",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": f"of {peak_kind}", "traffic": traffic,
