@@ -83,3 +83,35 @@ def test_sweep_weight_groupwise_g128(cq):
     torch.cuda.synchronize()
     parity.check_weight(W, "bf16", 4, scale=r.scale.cpu().numpy(), codes=r.codes.cpu().numpy(),
                         deq=bits_of(r.deq), zero_count=int(r.zero_count.item()), ref=ref)
+
+
+def test_diagnostics_operators_at_full_size(cq):
+    """Remove Kernel (with both kernel counts) and the Table 1 indicators on a full-size config."""
+    X, cfg = wl.activation("llama70b_attn")
+    Xd = to_dev(X, cfg.dtype)
+    want, removed, k_pt, k_cq = orc.remove_kernel(X, cfg.dtype, 0.15, 8, 1.0)
+    out, counts = cq.remove_kernel(Xd, 0.15, 8, 1.0)
+    torch.cuda.synchronize()
+    assert counts.cpu().tolist() == [removed, k_pt, k_cq]
+    assert np.array_equal(bits_of(out), want)
+    r = cq.quantize_act(Xd, 0.15, 8)
+    ref = orc.quantize_act(X, cfg.dtype, 0.15, 8, want_deq32=False, want_deq16=False)
+    assert tuple(cq.case_indicators(r).cpu().tolist()) == orc.case_indicators(ref.t, ref.c, ref.a, ref.b, 8)
+    assert int(r.zero_count.item()) == k_cq
+
+
+def test_crossquant_on_a_weight_matrix(cq):
+    """CrossQuant applied to weights (Appendix B: alpha_W = 0.55 for OPT-66B W4A4) is the activation entry point on W."""
+    W = wl.sweep_weight(0, 0)
+    Wd = to_dev(W, "bf16")
+    r = cq.quantize_act(Wd, 0.55, 4)
+    torch.cuda.synchronize()
+    parity.check_act(W, "bf16", 0.55, 4, t=r.t.cpu().numpy(), c=r.c.cpu().numpy(), a=r.row_scale.cpu().numpy(),
+                     b=r.col_scale.cpu().numpy(), codes=r.codes.cpu().numpy(), deq=bits_of(r.deq),
+                     zero_count=int(r.zero_count.item()))
+
+
+def test_no_bounded_wait_ever_gave_up(cq):
+    """Collected after the full-size runs: the staged quantize pass never abandoned a wait on a row copy."""
+    torch.cuda.synchronize()
+    assert cq.stage_fault() == 0
