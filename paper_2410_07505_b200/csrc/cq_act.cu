@@ -179,9 +179,13 @@ g1_absmax(const uint16_t* __restrict__ X, int64_t T, int64_t I, int64_t ld, int 
 }
 
 // ============================================================================ scale vectors
-// From the partial maxima of pass 1.  CTAs [0, col_ctas): 256 columns each; thread (vx, grp) reduces
-// every 8th partial row of vector column vx, shared memory combines the 8 groups, then one thread per
-// column.  CTAs [col_ctas, ...): one thread per row.
+// From the partial maxima of pass 1.  CTAs [0, col_ctas): 64 columns each; thread (vx, grp) reduces every
+// 32nd partial row of vector column vx (8 vector columns x 32 groups per CTA, so even the ~300 partial rows
+// of a narrow matrix cost each thread only ~10 independent loads), shared memory combines the 32 groups,
+// then one thread per column.  CTAs [col_ctas, ...): one thread per row.
+constexpr int kK2Cols = 8;       // vector columns per CTA
+constexpr int kK2Groups = 32;    // partial-row groups per CTA
+
 template <int DT>
 __global__ void __launch_bounds__(kThreads)
 k2_scales_from_partials(int64_t T, int64_t I, int I8, int nstrips, int Y, int col_ctas,
@@ -190,18 +194,18 @@ k2_scales_from_partials(int64_t T, int64_t I, int I8, int nstrips, int Y, int co
                         float* __restrict__ t_out, float* __restrict__ c_out,
                         float* __restrict__ a, float* __restrict__ b, float* __restrict__ ra, float* __restrict__ rb,
                         unsigned long long* __restrict__ zero_count) {
-    __shared__ uint4 s_part[8][32];
+    __shared__ uint4 s_part[kK2Groups][kK2Cols];
     const int tid = threadIdx.x;
     asm volatile("griddepcontrol.launch_dependents;");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (blockIdx.x == 0 && tid == 0 && zero_count != nullptr) *zero_count = 0ull;
     if (static_cast<int>(blockIdx.x) < col_ctas) {
-        const int vx = tid & 31, grp = tid >> 5;
-        const int vcol = blockIdx.x * 32 + vx;
+        const int vx = tid & (kK2Cols - 1), grp = tid / kK2Cols;
+        const int vcol = blockIdx.x * kK2Cols + vx;
         uint4 m = make_uint4(0, 0, 0, 0);
         if (vcol < I8) {
 #pragma unroll 4
-            for (int y = grp; y < Y; y += 8) {
+            for (int y = grp; y < Y; y += kK2Groups) {
                 const uint4 w = colpart[static_cast<int64_t>(y) * I8 + vcol];
                 m.x = max_u16x2(m.x, w.x); m.y = max_u16x2(m.y, w.y);
                 m.z = max_u16x2(m.z, w.z); m.w = max_u16x2(m.w, w.w);
@@ -209,12 +213,12 @@ k2_scales_from_partials(int64_t T, int64_t I, int I8, int nstrips, int Y, int co
         }
         s_part[grp][vx] = m;
         __syncthreads();
-        const int64_t j = static_cast<int64_t>(blockIdx.x) * 256 + tid;
-        if (j < I) {
+        const int64_t j = static_cast<int64_t>(blockIdx.x) * (kK2Cols * 8) + tid;
+        if (tid < kK2Cols * 8 && j < I) {
             const uint16_t* sp = reinterpret_cast<const uint16_t*>(&s_part[0][0]);
             uint32_t mx = 0;
 #pragma unroll
-            for (int k = 0; k < 8; ++k) mx = max(mx, static_cast<uint32_t>(sp[k * 256 + tid]));
+            for (int k = 0; k < kK2Groups; ++k) mx = max(mx, static_cast<uint32_t>(sp[k * (kK2Cols * 8) + tid]));
             const float cj = cvt16<DT>(static_cast<uint16_t>(mx));
             if (c_out != nullptr) c_out[j] = cj;
             float bj, rbj;
@@ -838,7 +842,7 @@ int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
         k2_scales_from_vectors<<<k2v_blocks, kThreads, 0, st>>>(T, I, t_given, c_given, alpha, qmax, a_dev, b_dev,
                                                                 ra_dev, rb_dev, zero_count);
     } else if (fast_in) {
-        const int col_ctas = (p.I8 + 31) / 32;
+        const int col_ctas = (p.I8 + kK2Cols - 1) / kK2Cols;
         const unsigned blocks = static_cast<unsigned>(col_ctas + (T + kThreads - 1) / kThreads);
         const uint4* cp4 = reinterpret_cast<const uint4*>(colpart);
         if (dtype == CQ_F16) {
