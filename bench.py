@@ -42,8 +42,8 @@ HOOK_EVERY = 8
 
 # DRAM traffic of the quantize pass from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum
 # per launch), valid only for the kernel sources whose digest is recorded with it.
-NCU_TRAFFIC = {"sources_sha256": "c355f682e4bf8899c8428f2ffe46ec6eb0ed8ab7fbad0d654be766130158b5d1",
-               "bytes_per_launch": 528244480}   # 235,183,616 read + 293,060,864 written
+NCU_TRAFFIC = {"sources_sha256": "18648882634bb6549f06a492afa05547557ffa127febf1d8601e8d29f514cef5",
+               "bytes_per_launch": 528703232}   # 235,232,768 read + 293,470,464 written
 
 
 def kernel_sources_digest() -> str:
