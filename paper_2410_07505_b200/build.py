@@ -14,7 +14,7 @@ LIB = os.path.join(HERE, "libcq.so")
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-fmad=false",            # no implicit FMA contraction: every rounding in the kernels is explicit
-    "-Xcompiler", "-fPIC", "-shared", "-Xptxas", "-v",
+    "-Xcompiler", "-fPIC", "-shared", "-Xptxas", "-v", "--threads", "0",
 ]
 
 

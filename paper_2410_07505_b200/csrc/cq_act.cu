@@ -479,121 +479,6 @@ g3_quantize(const uint16_t* __restrict__ X, int64_t T, int64_t I, int64_t ld, in
     if (zero_count != nullptr) cta_count_add(zeros, zero_count);
 }
 
-// ============================================================================ Remove Kernel
-// |fl32(x / s)| <= h decided from the reciprocal product where that is safe: v = x r differs from the
-// IEEE quotient by less than 2^-14.5 (|quotient| <= 128, all factors normal), so outside a band of
-// 2^-12 around h the comparison of |v| with h has the same outcome; inside it, or when a reciprocal
-// is the NaN marker of an extreme scale, the quotient itself is computed.
-__device__ __forceinline__ bool quotient_at_most(float x, float s, float r, float h, bool trusted) {
-    const float av = fabsf(__fmul_rn(x, r));
-    if (trusted && fabsf(av - h) > 0.000244140625f) return av <= h;
-    if (s == 0.0f) return true;
-    return fabsf(__fdiv_rn(x, s)) <= h;
-}
-
-// Same strip / resident-CTA layout as the quantize pass.  out = x with the elements of the kernel
-// replaced by +0; counts[0] += removed, counts[1] += |K| of per-token quantization, counts[2] += |K(CQ)|.
-template <int DT>
-__global__ void __launch_bounds__(kThreads)
-k9_remove_kernel(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
-                 const float* __restrict__ t, const float* __restrict__ a, const float* __restrict__ ra,
-                 const float* __restrict__ b, const float* __restrict__ rb, float qmaxf, float half_bound,
-                 uint4* __restrict__ out, unsigned long long* __restrict__ counts) {
-    const int tid = threadIdx.x, lane = tid & 31;
-    const int v = blockIdx.x * blockDim.x + tid;
-    const bool active = v < I8;
-    const int vv = active ? v : I8 - 1;
-    const int64_t ngroups = (T + 3) >> 2;
-    unsigned int n_removed = 0, n_pt = 0, n_cq = 0;
-    float bj[8], rbj[8];
-    {
-        const float4* bp = reinterpret_cast<const float4*>(b) + static_cast<int64_t>(vv) * 2;
-        const float4* rp = reinterpret_cast<const float4*>(rb) + static_cast<int64_t>(vv) * 2;
-        const float4 b0 = __ldg(bp), b1 = __ldg(bp + 1), q0 = __ldg(rp), q1 = __ldg(rp + 1);
-        bj[0] = b0.x; bj[1] = b0.y; bj[2] = b0.z; bj[3] = b0.w; bj[4] = b1.x; bj[5] = b1.y; bj[6] = b1.z; bj[7] = b1.w;
-        rbj[0] = q0.x; rbj[1] = q0.y; rbj[2] = q0.z; rbj[3] = q0.w; rbj[4] = q1.x; rbj[5] = q1.y; rbj[6] = q1.z; rbj[7] = q1.w;
-    }
-    for (int64_t g = blockIdx.y; g < ngroups; g += gridDim.y) {
-        // lanes 0-3: a_i of the four rows, 4-7: 1/a_i, 8-11: per-token scale t_i / qmax, 12-15: its reciprocal
-        float sv = 0.0f;
-        {
-            const int64_t row = min((g << 2) + (lane & 3), T - 1);
-            if (lane < 4) sv = __ldg(a + row);
-            else if (lane < 8) sv = __ldg(ra + row);
-            else if (lane < 16) {
-                const float spt = __fdiv_rn(__ldg(t + row), qmaxf);
-                sv = lane < 12 ? spt : guarded_rcp(spt);
-            }
-        }
-        uint4 w[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int64_t row = min((g << 2) + u, T - 1);
-            w[u] = ld_stream(X + row * ld8 + vv);
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int64_t row = (g << 2) + u;
-            const float au = __shfl_sync(0xFFFFFFFFu, sv, u), rau = __shfl_sync(0xFFFFFFFFu, sv, 4 + u);
-            const float spt = __shfl_sync(0xFFFFFFFFu, sv, 8 + u), rpt = __shfl_sync(0xFFFFFFFFu, sv, 12 + u);
-            if (row < T && active) {
-                uint32_t words[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const float2 x2 = unpack16x2<DT>(words[k]);
-                    const float xs[2] = {x2.x, x2.y};
-                    uint32_t keep_mask = 0xFFFFFFFFu;
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const int e = 2 * k + h;
-                        const float s = __fmul_rn(au, bj[e]), r = __fmul_rn(rau, rbj[e]);
-                        const bool trusted = r == r;
-                        const bool gone = quotient_at_most(xs[h], s, r, half_bound, trusted);
-                        n_removed += gone;
-                        n_cq += quotient_at_most(xs[h], s, r, 0.5f, trusted);
-                        n_pt += quotient_at_most(xs[h], spt, rpt, 0.5f, rpt == rpt);
-                        if (gone) keep_mask &= h ? 0x0000FFFFu : 0xFFFF0000u;
-                    }
-                    words[k] &= keep_mask;
-                }
-                st_stream(out + row * I8 + v, make_uint4(words[0], words[1], words[2], words[3]));
-            }
-        }
-    }
-    cta_count_add(n_removed, counts);
-    __syncthreads();
-    cta_count_add(n_pt, counts + 1);
-    __syncthreads();
-    cta_count_add(n_cq, counts + 2);
-}
-
-// General shapes / alignments: one thread per element, exact quotients.
-template <int DT>
-__global__ void __launch_bounds__(kThreads)
-g9_remove_kernel(const uint16_t* __restrict__ X, int64_t T, int64_t I, int64_t ld, const float* __restrict__ t,
-                 const float* __restrict__ a, const float* __restrict__ b, float qmaxf, float half_bound,
-                 uint16_t* __restrict__ out, unsigned long long* __restrict__ counts) {
-    const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-    unsigned int n_removed = 0, n_pt = 0, n_cq = 0;
-    if (idx < T * I) {
-        const int64_t i = idx / I, j = idx % I;
-        const uint16_t bits16 = X[i * ld + j];
-        const float x = cvt16<DT>(bits16);
-        const float s = __fmul_rn(a[i], b[j]), spt = __fdiv_rn(t[i], qmaxf);
-        const float nan = __int_as_float(0x7FC00000);
-        const bool gone = quotient_at_most(x, s, nan, half_bound, false);
-        n_removed = gone;
-        n_cq = quotient_at_most(x, s, nan, 0.5f, false);
-        n_pt = quotient_at_most(x, spt, nan, 0.5f, false);
-        out[idx] = gone ? static_cast<uint16_t>(0) : bits16;
-    }
-    cta_count_add(n_removed, counts);
-    __syncthreads();
-    cta_count_add(n_pt, counts + 1);
-    __syncthreads();
-    cta_count_add(n_cq, counts + 2);
-}
-
 // ============================================================================ host side
 static int g_tune_k1_ctas = 0;      // resident CTAs per SM assumed for pass 1 (0 = ask the runtime)
 static int g_tune_k3_ctas = 0;      // the same for pass 2
@@ -660,9 +545,9 @@ static bool fast_input(const void* X, int64_t I, int64_t ld) {
     return aligned(X, 16) && (I % 8 == 0) && (ld % 8 == 0);
 }
 
-static int launch_status() { return cudaGetLastError() == cudaSuccess ? CQ_OK : CQ_ERR_CUDA; }
+int launch_status() { return cudaGetLastError() == cudaSuccess ? CQ_OK : CQ_ERR_CUDA; }
 
-static int sm_count() {
+int sm_count() {
     int dev = 0, n = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
         n = 148;
@@ -787,6 +672,23 @@ static void launch_k3_deq(const Plan& p, const K3Args& k, int deq_mode, cudaStre
     if (deq_mode == 0) launch_k3_flags<DT, BITS, 0>(p, k, st);
     else if (deq_mode == 1) launch_k3_flags<DT, BITS, 1>(p, k, st);
     else launch_k3_flags<DT, BITS, 2>(p, k, st);
+}
+
+bool tuning_no_pdl() { return g_tune_no_pdl != 0; }
+
+// Scale vectors and their reciprocals into the workspace from finished t, c (for the diagnostics
+// kernels); *to_zero, if given, is cleared by the same launch.
+int scales_from_vectors(int64_t T, int64_t I, const float* t, const float* c, double alpha, int bits,
+                        void* workspace, size_t ws_bytes, unsigned long long* to_zero, cudaStream_t st) {
+    const Plan p = make_plan(T, I);
+    if (workspace == nullptr || !aligned(workspace, 256) || ws_bytes < p.total) return CQ_ERR_WORKSPACE;
+    char* ws = static_cast<char*>(workspace);
+    const unsigned blocks = static_cast<unsigned>((T + I + kThreads - 1) / kThreads);
+    k2_scales_from_vectors<<<blocks, kThreads, 0, st>>>(T, I, t, c, alpha, (1 << (bits - 1)) - 1,
+                                                        reinterpret_cast<float*>(ws + p.off_a), reinterpret_cast<float*>(ws + p.off_b),
+                                                        reinterpret_cast<float*>(ws + p.off_ra), reinterpret_cast<float*>(ws + p.off_rb),
+                                                        to_zero);
+    return launch_status();
 }
 
 // Shared body of cq_quantize_act and cq_kernel_count_x.  t_given/c_given: skip pass 1.
@@ -983,75 +885,6 @@ int cq_quantize_act(const void* X, int dtype, int64_t T, int64_t I, int64_t ld, 
     return cq::quantize_act_impl(X, dtype, T, I, ld, alpha, bits, nullptr, nullptr, t, c, row_scale, col_scale,
                                  codes, deq, deq_dtype, zero_count, workspace, workspace_bytes,
                                  static_cast<cudaStream_t>(stream));
-}
-
-int cq_kernel_count_x(const void* X, int dtype, int64_t T, int64_t I, int64_t ld, double alpha, int bits,
-                      const float* t, const float* c, unsigned long long* count,
-                      void* workspace, size_t workspace_bytes, void* stream) {
-    if (count == nullptr) return CQ_ERR_NULL;
-    if (T > 0 && I > 0 && (t == nullptr || c == nullptr)) return CQ_ERR_NULL;
-    return cq::quantize_act_impl(X, dtype, T, I, ld, alpha, bits, t, c, nullptr, nullptr, nullptr, nullptr,
-                                 nullptr, nullptr, dtype, count, workspace, workspace_bytes,
-                                 static_cast<cudaStream_t>(stream));
-}
-
-int cq_remove_kernel(const void* X, int dtype, int64_t T, int64_t I, int64_t ld, double alpha, int bits,
-                     float bound_scale, void* out, unsigned long long* counts,
-                     void* workspace, size_t workspace_bytes, void* stream) {
-    using namespace cq;
-    int rc = check_matrix(X, dtype, T, I, ld);
-    if (rc != CQ_OK) return rc;
-    if (bits != 4 && bits != 8) return CQ_ERR_BITS;
-    if (!(alpha >= 0.0 && alpha <= 1.0)) return CQ_ERR_ALPHA;
-    if (!(bound_scale >= 0.0f)) return CQ_ERR_SHAPE;
-    if (counts == nullptr) return CQ_ERR_NULL;
-    if ((reinterpret_cast<uintptr_t>(counts) % 8) != 0) return CQ_ERR_ALIGN;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (T == 0 || I == 0) {
-        return cudaMemsetAsync(counts, 0, 3 * sizeof(unsigned long long), st) == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
-    }
-    if (out == nullptr) return CQ_ERR_NULL;
-    if ((reinterpret_cast<uintptr_t>(out) % 2) != 0) return CQ_ERR_ALIGN;
-    // absmax pass and scale vectors into the workspace (no outputs requested: the quantize pass is skipped)
-    rc = quantize_act_impl(X, dtype, T, I, ld, alpha, bits, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr,
-                           nullptr, nullptr, dtype, nullptr, workspace, workspace_bytes, st);
-    if (rc != CQ_OK) return rc;
-    if (cudaMemsetAsync(counts, 0, 3 * sizeof(unsigned long long), st) != cudaSuccess) return CQ_ERR_CUDA;
-    const Plan p = make_plan(T, I);
-    char* ws = static_cast<char*>(workspace);
-    const float* t_dev = reinterpret_cast<const float*>(ws + p.off_t);
-    const float* a_dev = reinterpret_cast<const float*>(ws + p.off_a);
-    const float* b_dev = reinterpret_cast<const float*>(ws + p.off_b);
-    const float* ra_dev = reinterpret_cast<const float*>(ws + p.off_ra);
-    const float* rb_dev = reinterpret_cast<const float*>(ws + p.off_rb);
-    const float qmaxf = static_cast<float>((1 << (bits - 1)) - 1);
-    const float half_bound = 0.5f * bound_scale;
-    const bool fast = (reinterpret_cast<uintptr_t>(X) % 16) == 0 && (I % 8) == 0 && (ld % 8) == 0 &&
-                      (reinterpret_cast<uintptr_t>(out) % 16) == 0;
-    if (fast) {
-        int per_sm = 4;
-        int64_t y = static_cast<int64_t>(148) * per_sm / p.nstrips;
-        if (y > p.ngroups) y = p.ngroups;
-        if (y > 65535) y = 65535;
-        if (y < 1) y = 1;
-        const dim3 grid(p.nstrips, static_cast<unsigned>(y));
-        if (dtype == CQ_F16)
-            k9_remove_kernel<CQ_F16><<<grid, p.W, 0, st>>>(static_cast<const uint4*>(X), T, p.I8, ld / 8, t_dev, a_dev, ra_dev,
-                                                            b_dev, rb_dev, qmaxf, half_bound, static_cast<uint4*>(out), counts);
-        else
-            k9_remove_kernel<CQ_BF16><<<grid, p.W, 0, st>>>(static_cast<const uint4*>(X), T, p.I8, ld / 8, t_dev, a_dev, ra_dev,
-                                                             b_dev, rb_dev, qmaxf, half_bound, static_cast<uint4*>(out), counts);
-    } else {
-        const int64_t n = T * I;
-        const unsigned blocks = static_cast<unsigned>((n + kThreads - 1) / kThreads);
-        if (dtype == CQ_F16)
-            g9_remove_kernel<CQ_F16><<<blocks, kThreads, 0, st>>>(static_cast<const uint16_t*>(X), T, I, ld, t_dev, a_dev, b_dev,
-                                                                 qmaxf, half_bound, static_cast<uint16_t*>(out), counts);
-        else
-            g9_remove_kernel<CQ_BF16><<<blocks, kThreads, 0, st>>>(static_cast<const uint16_t*>(X), T, I, ld, t_dev, a_dev, b_dev,
-                                                                  qmaxf, half_bound, static_cast<uint16_t*>(out), counts);
-    }
-    return cudaGetLastError() == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
 }
 
 size_t cq_host_scratch_bytes(int64_t T, int64_t I, int bits, int want_codes, int want_deq, int deq_dtype) {

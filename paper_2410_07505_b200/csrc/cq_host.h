@@ -25,4 +25,10 @@ int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
                       void* codes, void* deq, int deq_dtype, unsigned long long* zero_count,
                       void* workspace, size_t ws_bytes, cudaStream_t st);
 
+int scales_from_vectors(int64_t T, int64_t I, const float* t, const float* c, double alpha, int bits,
+                        void* workspace, size_t ws_bytes, unsigned long long* to_zero, cudaStream_t st);
+int sm_count();
+int launch_status();
+bool tuning_no_pdl();     // programmatic dependent launch switched off through cq_set_tuning
+
 }  // namespace cq

@@ -211,7 +211,6 @@ k6_count_zero_codes(const uint8_t* __restrict__ codes, int bits, int64_t head, i
 }
 
 static bool aligned(const void* p, size_t n) { return (reinterpret_cast<uintptr_t>(p) % n) == 0; }
-static int launch_status() { return cudaGetLastError() == cudaSuccess ? CQ_OK : CQ_ERR_CUDA; }
 
 template <int DT, int BITS, int DEQ, bool CODES>
 static int launch_k4(int64_t R, int C8, int64_t ld8, const void* W, void* codes, float* scale, void* deq,
