@@ -843,7 +843,12 @@ int cq_set_tuning(const char* key, int value) {
 
 int cq_stage_fault(unsigned int* fault_host) {
     if (fault_host == nullptr) return CQ_ERR_NULL;
-    return cudaMemcpyFromSymbol(fault_host, cq::g_stage_fault, sizeof(unsigned int)) == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
+    unsigned int quantize_pass = 0, diagnostics = 0;
+    if (cudaMemcpyFromSymbol(&quantize_pass, cq::g_stage_fault, sizeof(unsigned int)) != cudaSuccess) return CQ_ERR_CUDA;
+    const int rc = cq::diag_stage_fault(&diagnostics);
+    if (rc != CQ_OK) return rc;
+    *fault_host = quantize_pass | diagnostics;
+    return CQ_OK;
 }
 
 int cq_set_timing_events(void* before_quantize_pass, void* after_quantize_pass) {

@@ -7,38 +7,58 @@
 #include "cq_host.h"
 
 #ifndef CQ_K9_MIN_CTAS
-#define CQ_K9_MIN_CTAS 2
+#define CQ_K9_MIN_CTAS 3
 #endif
 
 namespace cq {
 
-// |fl32(x / s)| <= h, decided from a reciprocal product where that is safe.  With every scale factor
-// in [2^-40, 2^40] the product v = x * (1/a_i) * (1/b_j) (or x * (1/s) for one scale) differs from the
-// real quotient z by less than 5 * 2^-24 |z|, and fl32(z) from z by at most 2^-24 |z|; so for h in
-// [2^-20, 2^20] (where nothing near h can be subnormal)
-//     |v| < h (1 - 2^-16)  =>  |fl32(z)| <  h,        |v| > h (1 + 2^-16)  =>  |fl32(z)| > h,
-// and only values inside that band (or a NaN, which fails both comparisons: the marker of an extreme
-// scale factor) need the quotient itself.  For h outside that range the band is (-1, inf): every
-// element takes the quotient.
-struct ZeroBand { float lo, hi; };
+// |fl32(x / s_ij)| <= h, decided without a division where that is safe.  With a_i, b_j in [2^-40, 2^40],
+// p = fl32(x * (1/b_j)) against the row's threshold m_i = fl32(h a_i) compares like |z| = |x / s_ij| against h
+// up to a relative error of 4 * 2^-24 (the roundings of 1/b_j, p, m_i and s_ij = fl32(a_i b_j)), and fl32(z)
+// lies within 2^-24 |z| of z; so for h in [2^-20, 2^20] (nothing near h can be subnormal) and
+// e_i = fl32(2^-18 h a_i), six times that error,
+//     |p| - m_i <= -e_i  =>  |fl32(z)| < h,        |p| - m_i >= e_i  =>  |fl32(z)| > h,
+// and only elements with | |p| - m_i | < e_i need the quotient itself.  Per-token quantization (one scale
+// per row, fl32(t_i / qmax)) compares |x| with fl32(t_i fl32(h / qmax)) in the same way (one more rounding).
+// A zero scale gives (m, e) = (inf, 0): everything in the row is in the kernel; a scale outside
+// [2^-40, 2^40], or h outside [2^-20, 2^20], gives (0, inf): every element takes the quotient.
+// f[]: what the row's scale (a_i, or t_i for per-token) is multiplied with to get m and e, in the order
+// CrossQuant with h = 1/2, per-token with h = 1/2, CrossQuant with the caller's bound.
+struct ZeroFactors { float f[6]; float inv_qmax; };
 
 static __device__ __noinline__ bool exact_at_most(float x, float s, float h) {
     if (s == 0.0f) return true;                       // the code of a zero scale is 0 by definition
     return fabsf(__fdiv_rn(x, s)) <= h;
 }
 
-// Same strip / resident-CTA layout and rolling four-row prefetch as the quantize pass; rows walked
-// from the last full group backwards, the ragged last group first by CTA y = 0.
+constexpr int kRing = 4;                           // stages of four rows per CTA
+__device__ unsigned int g_diag_stage_fault = 0;    // set if a bounded wait on a stage ever gave up
+
+// 0xFFFF in the low / high half of the result where d_lo / d_hi is negative (sign bit set), else 0:
+// byte permute in its sign-replicating mode on the top bytes of the two values.
+__device__ __forceinline__ uint32_t negative_halves(float d_lo, float d_hi) {
+    uint32_t r;
+    asm("prmt.b32 %0, %1, %2, 0xFFBB;" : "=r"(r) : "r"(__float_as_uint(d_lo)), "r"(__float_as_uint(d_hi)));
+    return r;
+}
+
+// Same strip / resident-CTA layout as the quantize pass, rows staged the same way: groups of four rows
+// arrive in a ring of shared-memory stages through asynchronous bulk copies issued by thread 0 (no
+// tensor map, no multicast; waits bounded, a wait that gives up raises g_diag_stage_fault).  Rows are
+// walked from the last full group backwards, the ragged last group first by CTA y = 0.
 //   WRITE: out = x, or +0 where |fl32(x / s_ij)| <= half_bound         (counts[0] += removed)
 //   DUAL : counts[1] += |K| of per-token quantization (scale fl32(t_i / qmax)), counts[2] += |K(CQ)|
 //   SAME : half_bound == 1/2, so "removed" and "in K(CQ)" are one test
 //   !WRITE && !DUAL: counts[0] += |K(CQ)| only
+// The comparisons are subtractions whose sign bits are gathered into per-row bit masks (one bit pair
+// per element pair): the masks give the output mask and the counts (popc); one chained comparison per
+// element collects whether any difference is inside the band, i.e. whether the row needs the quotients.
 template <int DT, bool WRITE, bool DUAL, bool SAME>
 __global__ void __launch_bounds__(kThreads, CQ_K9_MIN_CTAS)
 k9_zero_tests(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
-              const float* __restrict__ t, const float* __restrict__ a, const float* __restrict__ ra,
+              const float* __restrict__ t, const float* __restrict__ a,
               const float* __restrict__ b, const float* __restrict__ rb, float qmaxf,
-              float half_bound, ZeroBand band_h, ZeroBand band_half,
+              float half_bound, ZeroFactors zf,
               uint4* __restrict__ out, unsigned long long* __restrict__ counts) {
     const int tid = threadIdx.x, lane = tid & 31;
     const int v = blockIdx.x * blockDim.x + tid;
@@ -48,11 +68,13 @@ k9_zero_tests(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
     const int64_t nfull = T >> 2;
     const int64_t Y = gridDim.y;
     unsigned int n_removed = 0, n_pt = 0, n_cq = 0;
+    extern __shared__ __align__(128) unsigned char s_dyn[];
+    __shared__ uint64_t s_full[kRing];
 
     // the scale vectors come from the preceding kernel of the stream
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    if (warp_active) {
+    {
         float2 rb2[4];
         {
             const float4* rp = reinterpret_cast<const float4*>(rb) + static_cast<int64_t>(vv) * 2;
@@ -60,47 +82,44 @@ k9_zero_tests(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
             rb2[0] = make_float2(q0.x, q0.y); rb2[1] = make_float2(q0.z, q0.w);
             rb2[2] = make_float2(q1.x, q1.y); rb2[3] = make_float2(q1.z, q1.w);
         }
+        // a NaN among the column reciprocals (extreme b_j) sends all of this thread's vectors to the quotients
+        const bool cols_trusted = ((rb2[0].x + rb2[0].y) + (rb2[1].x + rb2[1].y)) +
+                                  ((rb2[2].x + rb2[2].y) + (rb2[3].x + rb2[3].y)) < INFINITY;
         const uint4* xp = X + vv;
 
-        auto do_row = [&](uint4& slot, const uint4* reload, bool has_next, float rau, float rpt, int64_t row, int vec) {
+        // thr[]: (m, e) of CrossQuant for 1/2, of per-token quantization, of CrossQuant for half_bound
+        auto do_row = [&](const uint4& slot, const float (&thr)[6], int64_t row, int vec) {
             const uint32_t words[4] = {slot.x, slot.y, slot.z, slot.w};
-            if (has_next) slot = ld_stream(reload);
-            const float2 ra2 = make_float2(rau, rau), rp2 = make_float2(rpt, rpt);
-            unsigned int r_rm = 0, r_pt = 0, r_cq = 0;
-            bool undecided = false;
+            uint32_t m_c = 0, m_p = 0, m_g = 0;
+            bool undecided = !cols_trusted;
             uint32_t ow[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
+                const uint32_t bit = 0x00010001u << k;
                 const float2 x = unpack16x2<DT>(words[k]);
-                const float2 vq = __fmul2_rn(x, __fmul2_rn(ra2, rb2[k]));
-                const float av[2] = {fabsf(vq.x), fabsf(vq.y)};
-                uint32_t keep = 0xFFFFFFFFu;
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const bool z = av[h] < band_half.lo, nz = av[h] > band_half.hi;
-                    r_cq += z;
-                    undecided |= !(z || nz);
-                    bool gone = z;
-                    if constexpr (!SAME) {
-                        const bool g = av[h] < band_h.lo, ng = av[h] > band_h.hi;
-                        undecided |= !(g || ng);
-                        gone = g;
-                    }
-                    r_rm += gone;
-                    if (gone) keep &= h ? 0x0000FFFFu : 0xFFFF0000u;
+                const float2 p = __fmul2_rn(x, rb2[k]);
+                const float px = fabsf(p.x), py = fabsf(p.y);
+                const float d0 = __fadd_rn(px, -thr[0]), d1 = __fadd_rn(py, -thr[0]);
+                undecided |= fabsf(d0) < thr[1];
+                undecided |= fabsf(d1) < thr[1];
+                uint32_t gone = negative_halves(d0, d1);
+                m_c |= gone & bit;
+                if constexpr (!SAME) {
+                    const float g0 = __fadd_rn(px, -thr[4]), g1 = __fadd_rn(py, -thr[4]);
+                    undecided |= fabsf(g0) < thr[5];
+                    undecided |= fabsf(g1) < thr[5];
+                    gone = negative_halves(g0, g1);
+                    m_g |= gone & bit;
                 }
                 if constexpr (DUAL) {
-                    const float2 vp = __fmul2_rn(x, rp2);
-                    const float ap[2] = {fabsf(vp.x), fabsf(vp.y)};
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const bool z = ap[h] < band_half.lo, nz = ap[h] > band_half.hi;
-                        r_pt += z;
-                        undecided |= !(z || nz);
-                    }
+                    const float e0 = __fadd_rn(fabsf(x.x), -thr[2]), e1 = __fadd_rn(fabsf(x.y), -thr[2]);
+                    undecided |= fabsf(e0) < thr[3];
+                    undecided |= fabsf(e1) < thr[3];
+                    m_p |= negative_halves(e0, e1) & bit;
                 }
-                ow[k] = words[k] & keep;
+                ow[k] = words[k] & ~gone;
             }
+            unsigned int r_cq = __popc(m_c), r_pt = __popc(m_p), r_rm = SAME ? r_cq : __popc(m_g);
             if (undecided) {
                 // Rare: some element sits within 2^-16 (relative) of a bound, or a scale factor is extreme.
                 // The whole vector is decided again from the IEEE quotients.
@@ -108,7 +127,7 @@ k9_zero_tests(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
                 const float ai = __ldg(a + row);
                 const float spt = DUAL ? __fdiv_rn(__ldg(t + row), qmaxf) : 0.0f;
                 const float* bp = b + static_cast<int64_t>(vv) * 8;
-#pragma unroll 1
+#pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     const float2 x = unpack16x2<DT>(words[k]);
                     const float xs[2] = {x.x, x.y};
@@ -131,49 +150,84 @@ k9_zero_tests(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
                 if (active) st_stream(out + vec, make_uint4(ow[0], ow[1], ow[2], ow[3]));
             }
         };
-        // lanes 0-3: 1/a_i of a group's four rows; lanes 4-7: reciprocal of the per-token scale t_i / qmax
-        auto load_scales = [&](int64_t g) {
+        // Lane l holds threshold number l / 4 (order of thr[] above) of row l % 4 of the group.  The scale is
+        // fetched one group ahead (load_scale) and turned into the threshold when its group comes up.
+        constexpr int kKinds = !DUAL ? 2 : (SAME ? 4 : 6);
+        const int kind = lane >> 2;
+        const bool per_token = kind == 2 || kind == 3;
+        const bool is_mid = (kind & 1) == 0;
+        float factor = zf.f[0];
+#pragma unroll
+        for (int k = 1; k < kKinds; ++k) factor = kind == k ? zf.f[k] : factor;
+        auto load_scale = [&](int64_t g) {
+            if (kind >= kKinds) return 0.0f;
             const int64_t row = min((g << 2) + (lane & 3), T - 1);
-            float sv = 0.0f;
-            if (lane < 4) sv = __ldg(ra + row);
-            else if (DUAL && lane < 8) sv = guarded_rcp(__fdiv_rn(__ldg(t + row), qmaxf));
-            return sv;
+            return per_token ? __ldg(t + row) : __ldg(a + row);
+        };
+        auto threshold_of = [&](float raw) {
+            const float sc = (DUAL && per_token) ? __fmul_rn(raw, zf.inv_qmax) : raw;      // range check only
+            if (raw == 0.0f) return is_mid ? INFINITY : 0.0f;
+            if (sc >= kScaleLo && sc <= kScaleHi) return __fmul_rn(factor, raw);
+            return is_mid ? 0.0f : INFINITY;
+        };
+        auto row_thresholds = [&](float tv, int u, float (&thr)[6]) {
+#pragma unroll
+            for (int k = 0; k < 6; ++k) thr[k] = k < kKinds ? __shfl_sync(0xFFFFFFFFu, tv, 4 * k + u) : 0.0f;
         };
 
-        if ((T & 3) != 0 && blockIdx.y == 0) {                           // ragged last group
-            const float sv = load_scales(nfull);
+        if ((T & 3) != 0 && blockIdx.y == 0 && warp_active) {            // ragged last group
+            const float tv = threshold_of(load_scale(nfull));
             for (int u = 0; u < static_cast<int>(T & 3); ++u) {
                 const int64_t row = (nfull << 2) + u;
-                uint4 slot = ld_stream(xp + row * ld8);
-                do_row(slot, nullptr, false, __shfl_sync(0xFFFFFFFFu, sv, u), __shfl_sync(0xFFFFFFFFu, sv, 4 + u), row,
-                       static_cast<int>(row * I8 + vv));
+                const uint4 slot = ld_stream(xp + row * ld8);
+                float thr[6];
+                row_thresholds(tv, u, thr);
+                do_row(slot, thr, row, static_cast<int>(row * I8 + vv));
             }
         }
 
-        int64_t pos = blockIdx.y;
-        if (pos < nfull) {
-            int64_t g = nfull - 1 - pos;
-            const int64_t xstep = -4 * Y * ld8;
-            const int ostep = static_cast<int>(-4 * Y * I8);
-            const uint4* p = xp + (g << 2) * ld8;
-            int vec = static_cast<int>((g << 2) * I8 + vv);
-            uint4 w[4];
+        uint4* stage = reinterpret_cast<uint4*>(s_dyn);                   // [kRing][4 rows][blockDim.x]
+        const int Wv = blockDim.x;
+        const int strip0 = blockIdx.x * Wv;
+        const uint32_t seg_bytes = static_cast<uint32_t>(min(Wv, I8 - strip0)) * 16u;
+        const int64_t first = blockIdx.y;
+        const int64_t mine = first < nfull ? (nfull - first + Y - 1) / Y : 0;          // groups of this CTA
+        auto group_at = [&](int64_t k) { return nfull - 1 - (first + k * Y); };
+        auto issue = [&](int64_t k) {                                     // thread 0 only
+            if (k >= mine) return;
+            const int st = static_cast<int>(k % kRing);
+            const uint4* src = X + (group_at(k) << 2) * ld8 + strip0;
+            mbar_expect_tx(&s_full[st], 4u * seg_bytes);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) w[u] = ld_stream(p + u * ld8);
-            float sv = load_scales(g);
-            for (; pos < nfull; pos += Y) {
-                const bool has_next = pos + Y < nfull;
-                const uint4* pn = p + xstep;
-                float svn = 0.0f;
-                if (has_next) svn = load_scales(g - Y);
+            for (int u = 0; u < 4; ++u) bulk_load(stage + (st * 4 + u) * Wv, src + u * ld8, seg_bytes, &s_full[st]);
+        };
+        if (tid == 0) {
 #pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    do_row(w[u], pn + u * ld8, has_next, __shfl_sync(0xFFFFFFFFu, sv, u), __shfl_sync(0xFFFFFFFFu, sv, 4 + u),
-                           (g << 2) + u, vec + u * I8);
-                p = pn;
-                vec += ostep;
-                g -= Y;
-                sv = svn;
+            for (int st = 0; st < kRing; ++st) mbar_init(&s_full[st], 1);
+            mbar_init_fence();
+        }
+        __syncthreads();
+        if (tid == 0) {
+            for (int k = 0; k < kRing - 1; ++k) issue(k);
+        }
+        float raw = mine > 0 ? load_scale(group_at(0)) : 0.0f;
+        for (int64_t k = 0; k < mine; ++k) {
+            const int64_t g = group_at(k);
+            const float tv = threshold_of(raw);
+            if (k + 1 < mine) raw = load_scale(group_at(k + 1));
+            __syncthreads();                                              // everybody is done with group k-1: its stage is free
+            if (tid == 0) issue(k + kRing - 1);
+            const int st = static_cast<int>(k % kRing);
+            if (!mbar_wait(&s_full[st], static_cast<uint32_t>((k / kRing) & 1))) atomicExch(&g_diag_stage_fault, 1u);
+            if (warp_active) {
+                const int vec = static_cast<int>((g << 2) * I8 + vv);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const uint4 cur = stage[(st * 4 + u) * Wv + tid];
+                    float thr[6];
+                    row_thresholds(tv, u, thr);
+                    do_row(cur, thr, (g << 2) + u, vec + u * I8);
+                }
             }
         }
         if (!active) { n_removed = 0; n_pt = 0; n_cq = 0; }
@@ -223,21 +277,33 @@ g9_zero_tests(const uint16_t* __restrict__ X, int64_t T, int64_t I, int64_t ld, 
 }
 
 // ============================================================================ host side
-static ZeroBand band_of(float h) {
-    if (h >= 9.5367431640625e-07f && h <= 1048576.0f)                 // [2^-20, 2^20]
-        return ZeroBand{h * (1.0f - 1.52587890625e-05f), h * (1.0f + 1.52587890625e-05f)};
-    return ZeroBand{-1.0f, INFINITY};
+static ZeroFactors factors_of(float h, float qmaxf) {
+    auto pair = [](float bound, float div, float* out) {
+        if (bound >= 9.5367431640625e-07f && bound <= 1048576.0f) {   // [2^-20, 2^20]
+            out[0] = bound / div;
+            out[1] = bound * 3.814697265625e-06f / div;               // 2^-18
+        } else {
+            out[0] = 0.0f;
+            out[1] = INFINITY;
+        }
+    };
+    ZeroFactors z{};
+    pair(0.5f, 1.0f, z.f);
+    pair(0.5f, qmaxf, z.f + 2);
+    pair(h, 1.0f, z.f + 4);
+    z.inv_qmax = 1.0f / qmaxf;
+    return z;
 }
 
 template <typename... KArgs, typename... Args>
-static void launch_after(void (*kern)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+static void launch_after(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = tuning_no_pdl() ? 0 : 1;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = grid;
     cfg.blockDim = block;
-    cfg.dynamicSmemBytes = 0;
+    cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
@@ -252,26 +318,33 @@ struct ZeroArgs {
 };
 
 template <int DT, bool WRITE, bool DUAL, bool SAME>
-static void launch_k9(const Plan& p, const ZeroArgs& z, cudaStream_t st) {
+static bool launch_k9(const Plan& p, const ZeroArgs& z, cudaStream_t st) {
     auto kern = k9_zero_tests<DT, WRITE, DUAL, SAME>;
+    const size_t smem = static_cast<size_t>(kRing) * 4 * p.W * 16;
     int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, p.W, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, p.W, smem) != cudaSuccess || per_sm < 1) {
+        cudaGetLastError();
+        return false;
+    }
     int64_t y = static_cast<int64_t>(sm_count()) * per_sm / p.nstrips;
     if (y > p.ngroups) y = p.ngroups;
     if (y > 65535) y = 65535;
     if (y < 1) y = 1;
-    launch_after(kern, dim3(p.nstrips, static_cast<unsigned>(y)), dim3(p.W), st, static_cast<const uint4*>(z.X), z.T, p.I8,
-                 z.ld / 8, z.t, z.a, z.ra, z.b, z.rb, z.qmaxf, z.half_bound, band_of(z.half_bound), band_of(0.5f),
+    launch_after(kern, dim3(p.nstrips, static_cast<unsigned>(y)), dim3(p.W), smem, st, static_cast<const uint4*>(z.X), z.T,
+                 p.I8, z.ld / 8, z.t, z.a, z.b, z.rb, z.qmaxf, z.half_bound, factors_of(z.half_bound, z.qmaxf),
                  static_cast<uint4*>(z.out), z.counts);
+    return true;
 }
 
 template <int DT>
 static void launch_zero_tests(const Plan& p, const ZeroArgs& z, bool only_cq, bool fast, cudaStream_t st) {
     if (fast) {
-        if (only_cq) launch_k9<DT, false, false, true>(p, z, st);
-        else if (z.half_bound == 0.5f) launch_k9<DT, true, true, true>(p, z, st);
-        else launch_k9<DT, true, true, false>(p, z, st);
-    } else {
+        if (only_cq) fast = launch_k9<DT, false, false, true>(p, z, st);
+        else if (z.half_bound == 0.5f) fast = launch_k9<DT, true, true, true>(p, z, st);
+        else fast = launch_k9<DT, true, true, false>(p, z, st);
+    }
+    if (!fast) {
         const int64_t n = z.T * z.I;
         const unsigned blocks = static_cast<unsigned>((n + kThreads - 1) / kThreads);
         g9_zero_tests<DT><<<blocks, kThreads, 0, st>>>(static_cast<const uint16_t*>(z.X), z.T, z.I, z.ld, z.t, z.a, z.b,
@@ -294,6 +367,10 @@ static ZeroArgs zero_args(const Plan& p, void* workspace, const void* X, int64_t
 // vectors of 8 columns are indexed with 32-bit integers in the tiled kernel
 static bool fast_shape(const Plan& p, const void* X, int64_t T, int64_t I, int64_t ld) {
     return is_aligned(X, 16) && (I % 8) == 0 && (ld % 8) == 0 && T * static_cast<int64_t>(p.I8) < (int64_t(1) << 31);
+}
+
+int diag_stage_fault(unsigned int* fault_host) {
+    return cudaMemcpyFromSymbol(fault_host, g_diag_stage_fault, sizeof(unsigned int)) == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
 }
 
 }  // namespace cq

@@ -29,6 +29,7 @@ int scales_from_vectors(int64_t T, int64_t I, const float* t, const float* c, do
                         void* workspace, size_t ws_bytes, unsigned long long* to_zero, cudaStream_t st);
 int sm_count();
 int launch_status();
+int diag_stage_fault(unsigned int* fault_host);   // flag of the staged diagnostics kernels
 bool tuning_no_pdl();     // programmatic dependent launch switched off through cq_set_tuning
 
 }  // namespace cq
