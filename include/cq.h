@@ -166,7 +166,8 @@ int cq_kernel_count_x(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
  *   W in device [R x ld]; codes out int8[R*C] or packed uint8[R*C/2]; scale out float[R];
  *   deq out [R*C] of deq_dtype (W's dtype or CQ_F32); zero_count out device uint64.
  *   codes, scale, deq, zero_count are nullable.  Each row is read from HBM once while it fits
- *   in shared memory (C <= 110,592), twice otherwise.
+ *   in shared memory (C <= 110,592), twice otherwise; rows of 32 KB or more arrive through one
+ *   asynchronous bulk copy each.
  */
 int cq_quantize_weight_per_channel(const void* W, int dtype, int64_t R, int64_t C, int64_t ld, int bits,
                                    void* codes, float* scale, void* deq, int deq_dtype,
@@ -216,7 +217,8 @@ int cq_case_indicators(const float* t, const float* c, const float* row_scale, c
  * Returns CQ_OK or CQ_ERR_SHAPE. */
 int cq_set_tuning(const char* key, int value);
 
-/* Health check.  The quantize pass waits for its asynchronous row copies with a bounded number of polls;
+/* Health check.  The quantize pass, the diagnostics passes (cq_remove_kernel, cq_kernel_count_x) and the
+ * weight quantizer on long rows wait for their asynchronous row copies with a bounded number of polls;
  * if a wait ever gives up, a device flag is raised (results of that call are then undefined).  This
  * copies the flag of the current device to *fault_host (0 = never happened).  Synchronises the device. */
 int cq_stage_fault(unsigned int* fault_host);

@@ -675,6 +675,7 @@ static void launch_k3_deq(const Plan& p, const K3Args& k, int deq_mode, cudaStre
 }
 
 bool tuning_no_pdl() { return g_tune_no_pdl != 0; }
+bool tuning_no_stage() { return g_tune_no_stage != 0; }
 
 // Scale vectors and their reciprocals into the workspace from finished t, c (for the diagnostics
 // kernels); *to_zero, if given, is cleared by the same launch.
@@ -843,11 +844,12 @@ int cq_set_tuning(const char* key, int value) {
 
 int cq_stage_fault(unsigned int* fault_host) {
     if (fault_host == nullptr) return CQ_ERR_NULL;
-    unsigned int quantize_pass = 0, diagnostics = 0;
+    unsigned int quantize_pass = 0, diagnostics = 0, weights = 0;
     if (cudaMemcpyFromSymbol(&quantize_pass, cq::g_stage_fault, sizeof(unsigned int)) != cudaSuccess) return CQ_ERR_CUDA;
-    const int rc = cq::diag_stage_fault(&diagnostics);
+    int rc = cq::diag_stage_fault(&diagnostics);
+    if (rc == CQ_OK) rc = cq::weight_stage_fault(&weights);
     if (rc != CQ_OK) return rc;
-    *fault_host = quantize_pass | diagnostics;
+    *fault_host = quantize_pass | diagnostics | weights;
     return CQ_OK;
 }
 

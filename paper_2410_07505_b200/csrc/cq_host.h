@@ -30,6 +30,8 @@ int scales_from_vectors(int64_t T, int64_t I, const float* t, const float* c, do
 int sm_count();
 int launch_status();
 int diag_stage_fault(unsigned int* fault_host);   // flag of the staged diagnostics kernels
+int weight_stage_fault(unsigned int* fault_host); // flag of the bulk-copy weight kernel
+bool tuning_no_stage();   // staged (bulk-copy) variants switched off through cq_set_tuning
 bool tuning_no_pdl();     // programmatic dependent launch switched off through cq_set_tuning
 
 }  // namespace cq

@@ -10,7 +10,11 @@ constexpr int kMaxSmemRowBytes = 221184;   // 216 KB of the 227 KB a CTA may use
 // ============================================================================ weight rows
 // One CTA per stored row.  The row is read from HBM once into shared memory while its absolute
 // maximum is reduced; each thread later quantizes exactly the vectors it staged itself.
-template <int DT, int BITS, int DEQ, bool CODES>
+// BULK (long rows, of which only a few CTAs fit on an SM): the row arrives through one asynchronous bulk
+// copy issued by thread 0, so the whole row is in flight at once instead of four vectors per thread.
+__device__ unsigned int g_weight_stage_fault = 0;   // set if the bounded wait on a row copy ever gave up
+
+template <int DT, int BITS, int DEQ, bool CODES, bool BULK>
 __global__ void __launch_bounds__(kThreads)
 k4_weight_rows(const uint4* __restrict__ W, int C8, int64_t ld8,
                void* __restrict__ codes, float* __restrict__ scale, void* __restrict__ deq,
@@ -23,12 +27,32 @@ k4_weight_rows(const uint4* __restrict__ W, int C8, int64_t ld8,
     const uint4* p = W + row * ld8;
 
     uint32_t mm = 0;
+    if constexpr (BULK) {
+        __shared__ uint64_t s_bar;
+        if (tid == 0) {
+            mbar_init(&s_bar, 1);
+            mbar_init_fence();
+        }
+        __syncthreads();
+        if (tid == 0) {
+            mbar_expect_tx(&s_bar, static_cast<uint32_t>(C8) * 16u);
+            bulk_load(s_vec, p, static_cast<uint32_t>(C8) * 16u, &s_bar);
+        }
+        if (!mbar_wait(&s_bar, 0u)) atomicExch(&g_weight_stage_fault, 1u);
 #pragma unroll 4
-    for (int v = tid; v < C8; v += kThreads) {
-        uint4 w = ld_stream(p + v);
-        s_vec[v] = w;
-        mm = max_u16x2(mm, max_u16x2(max_u16x2(w.x & 0x7FFF7FFFu, w.y & 0x7FFF7FFFu),
-                                     max_u16x2(w.z & 0x7FFF7FFFu, w.w & 0x7FFF7FFFu)));
+        for (int v = tid; v < C8; v += kThreads) {
+            const uint4 w = s_vec[v];
+            mm = max_u16x2(mm, max_u16x2(max_u16x2(w.x & 0x7FFF7FFFu, w.y & 0x7FFF7FFFu),
+                                         max_u16x2(w.z & 0x7FFF7FFFu, w.w & 0x7FFF7FFFu)));
+        }
+    } else {
+#pragma unroll 4
+        for (int v = tid; v < C8; v += kThreads) {
+            uint4 w = ld_stream(p + v);
+            s_vec[v] = w;
+            mm = max_u16x2(mm, max_u16x2(max_u16x2(w.x & 0x7FFF7FFFu, w.y & 0x7FFF7FFFu),
+                                         max_u16x2(w.z & 0x7FFF7FFFu, w.w & 0x7FFF7FFFu)));
+        }
     }
     uint32_t m16 = __reduce_max_sync(0xFFFFFFFFu, max(mm & 0xFFFFu, mm >> 16));
     if (lane == 0) s_max[warp] = m16;
@@ -216,7 +240,9 @@ template <int DT, int BITS, int DEQ, bool CODES>
 static int launch_k4(int64_t R, int C8, int64_t ld8, const void* W, void* codes, float* scale, void* deq,
                      unsigned long long* zc, cudaStream_t st) {
     const size_t smem = static_cast<size_t>(C8) * 16;
-    auto kern = k4_weight_rows<DT, BITS, DEQ, CODES>;
+    // rows of 32 KB or more leave room for at most seven CTAs per SM: those take the bulk-copy variant
+    const bool bulk = smem >= 32 * 1024 && !tuning_no_stage();
+    auto kern = bulk ? k4_weight_rows<DT, BITS, DEQ, CODES, true> : k4_weight_rows<DT, BITS, DEQ, CODES, false>;
     if (smem > 48 * 1024) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
             return CQ_ERR_CUDA;
@@ -236,6 +262,10 @@ static int launch_k4_out(int deq_mode, bool has_codes, int64_t R, int C8, int64_
     if (deq_mode == 0) return launch_k4<DT, BITS, 0, false>(R, C8, ld8, W, codes, scale, deq, zc, st);
     if (deq_mode == 1) return launch_k4<DT, BITS, 1, false>(R, C8, ld8, W, codes, scale, deq, zc, st);
     return launch_k4<DT, BITS, 2, false>(R, C8, ld8, W, codes, scale, deq, zc, st);
+}
+
+int weight_stage_fault(unsigned int* fault_host) {
+    return cudaMemcpyFromSymbol(fault_host, g_weight_stage_fault, sizeof(unsigned int)) == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
 }
 
 }  // namespace cq
