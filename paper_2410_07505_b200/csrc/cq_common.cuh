@@ -17,6 +17,7 @@ constexpr uint32_t kMagicBits = 0x4B400000u;
 // 1/2 - 2^-16: a candidate code q is accepted without the IEEE division when |x - q s| < s * kHalfMinus.
 constexpr float kHalfMinus = 0.4999847412109375f;
 
+constexpr float kScaleLoTie = 2.350988701644575e-38f;    // 2^-125: s / 2 is a normal number, hence exact, from here up
 constexpr int kThreads = 256;      // largest CTA of the tiled kernels
 constexpr int kMaxRowsPerCta = 128;
 
@@ -112,12 +113,12 @@ __device__ __forceinline__ uint16_t pack16(float v) {
 // equal to round-half-even(fl32(x / s)): with z = x/s and |z| <= 128, fl32(z) lies within 2^-17 of
 // z, so |z - q| < 1/2 - 2^-16 (checked on the exactly computed residual x - q s) forces the IEEE
 // quotient to round to q as well.  Any NaN or infinity in the candidate makes the test fail.
-__device__ __forceinline__ float quant_candidate(float x, float s, float r, float qmaxf, bool& ok) {
+__device__ __forceinline__ float quant_candidate(float x, float s, float r, float qmaxf, bool& ok, float& e) {
     float v = __fmul_rn(x, r);
     v = fminf(fmaxf(v, -qmaxf), qmaxf);
     float y = __fadd_rn(v, kMagic);
     float qf = __fadd_rn(y, -kMagic);
-    float e = __fmaf_rn(-qf, s, x);
+    e = __fmaf_rn(-qf, s, x);
     ok = fabsf(e) < __fmul_rn(s, kHalfMinus);
     return y;
 }
@@ -131,6 +132,26 @@ static __device__ __noinline__ float quant_exact(float x, float s, float qmaxf) 
     return __fadd_rn(q, kMagic);        // (-0) + kMagic == kMagic
 }
 
+// For a candidate that failed its test.  First the exact tie: if the candidate's residual e = x - q s is
+// exactly +-s/2, then x / s = q +- 1/2 (for q != 0 up to a relative 2^-24 of the 1/2, which fl32 absorbs),
+// the IEEE quotient is that half-integer and round-half-even picks the even one of q and q +- 1.  16-bit
+// inputs make such ties common (a weight row whose maximum has the mantissa 2 * 127 puts a quarter of
+// its elements on one), so they are settled without the division.  Everything else takes quant_exact.
+// y = kMagic + q with a finite q; s / 2 is exact for s >= 2^-125.
+static __device__ __noinline__ float quant_settle(float x, float s, float qmaxf, float y, float e) {
+    if (s >= kScaleLoTie && fabsf(e) == __fmul_rn(s, 0.5f)) {
+        float qf = __fadd_rn(y, -kMagic);
+        if ((__float_as_uint(y) & 1u) != 0u) qf = __fadd_rn(qf, e > 0.0f ? 1.0f : -1.0f);   // q odd: step to the even side
+        qf = fminf(fmaxf(qf, -qmaxf), qmaxf);
+        return __fadd_rn(qf, kMagic);
+    }
+    if (s == 0.0f) return kMagic;
+    float u = __fdiv_rn(x, s);
+    float q = rintf(u);
+    q = fminf(fmaxf(q, -qmaxf), qmaxf);
+    return __fadd_rn(q, kMagic);
+}
+
 // ---- eight elements of one row -------------------------------------------------------------
 // Scale factors outside [2^-40, 2^40] get a NaN "reciprocal"; callers test for it (x != x) and send
 // such rows / columns to the defining sequence.  A factor of exactly zero means the whole row or
@@ -141,6 +162,15 @@ constexpr float kScaleHi = 1.099511627776e12f;         // 2^40
 __device__ __forceinline__ float guarded_rcp(float f) {
     if (f == 0.0f) return 0.0f;
     return (f >= kScaleLo && f <= kScaleHi) ? __fdiv_rn(1.0f, f) : __int_as_float(0x7FC00000);
+}
+// Same contract from the hardware's approximate reciprocal (relative error at most 2^-23 on normal
+// inputs): for kernels that need one reciprocal per small group, where the exact one would dominate.
+// The candidate built from it is x * r with two roundings, 3 * 2^-24 in all: inside the bound below.
+__device__ __forceinline__ float guarded_rcp_approx(float f) {
+    if (f == 0.0f) return 0.0f;
+    float r;
+    asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(f));
+    return (f >= kScaleLo && f <= kScaleHi) ? r : __int_as_float(0x7FC00000);
 }
 // The candidate q = round-half-even(v), v = x * (1/a_i) * (1/b_j), is accepted when |v - q| < 1/2 - 2^-12.
 // With a_i, b_j in [2^-40, 2^40] they, their reciprocals, s_ij = fl32(a_i b_j) and the reciprocal product
@@ -153,7 +183,7 @@ constexpr float kAcceptBelow = 0.499755859375f;         // 1/2 - 2^-12
 // y2[k] = kMagic + q and q2[k] = q for elements 2k, 2k+1.  UNIFORM: one scale `a` for the whole row
 // (b2, rb2 unused).  `trusted`: none of the reciprocals involved is the NaN marker (a NaN would not
 // survive the max below, so it has to be tested where the reciprocals are loaded).
-template <int DT, int BITS, bool UNIFORM>
+template <int DT, int BITS, bool UNIFORM, bool LEAN = false>
 __device__ __forceinline__ void quantize_row8(const uint4& w, float a, float ra, const float2 (&b2)[4],
                                               const float2 (&rb2)[4], bool trusted,
                                               float2 (&y2)[4], float2 (&q2)[4]) {
@@ -174,22 +204,31 @@ __device__ __forceinline__ void quantize_row8(const uint4& w, float a, float ra,
         worst = fmaxf(fmaxf(worst, fabsf(f.x)), fabsf(f.y));
     }
     if (!(trusted && worst < kAcceptBelow)) {
-        // Rare: some element is too close to a rounding boundary (or a scale factor is extreme) for the
-        // cheap test to decide.  Re-examine each element with the exact residual; the undecided ones
-        // take the defining sequence (IEEE division, round half to even, clamp).
+        // Some element is too close to a rounding boundary (or a scale factor is extreme) for the cheap
+        // test to decide.  The pairs that hold such an element are found again; their elements are
+        // re-examined with the exact residual, and the undecided ones are settled as exact ties or take
+        // the defining sequence (IEEE division, round half to even, clamp).  LEAN re-examines all eight
+        // elements instead: no fast result has to survive this region, which saves the registers a
+        // kernel that lives on occupancy needs.
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             const float2 x = unpack16x2<DT>(words[k]);
+            const float2 r = UNIFORM ? ra2 : __fmul2_rn(ra2, rb2[k]);
+            if constexpr (!LEAN) {
+                const float2 f = __ffma2_rn(q2[k], neg1, __fmul2_rn(x, r));
+                if (trusted && fmaxf(fabsf(f.x), fabsf(f.y)) < kAcceptBelow) continue;
+            }
             const float xs[2] = {x.x, x.y};
             const float bs[2] = {UNIFORM ? 1.0f : b2[k].x, UNIFORM ? 1.0f : b2[k].y};
-            const float rs[2] = {UNIFORM ? 1.0f : rb2[k].x, UNIFORM ? 1.0f : rb2[k].y};
+            const float rs[2] = {r.x, r.y};
             float ys[2];
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const float sh = UNIFORM ? a : __fmul_rn(a, bs[h]);
                 bool good;
-                ys[h] = quant_candidate(xs[h], sh, UNIFORM ? ra : __fmul_rn(ra, rs[h]), qmaxf, good);
-                if (!good) ys[h] = quant_exact(xs[h], sh, qmaxf);
+                float e;
+                ys[h] = quant_candidate(xs[h], sh, rs[h], qmaxf, good, e);
+                if (!good) ys[h] = quant_settle(xs[h], sh, qmaxf, ys[h], e);
             }
             y2[k] = make_float2(ys[0], ys[1]);
             q2[k] = __fadd2_rn(y2[k], nm2);

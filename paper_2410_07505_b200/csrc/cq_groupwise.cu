@@ -17,26 +17,57 @@ k7_weight_groups(const uint4* __restrict__ W, int64_t nvec, int C8, int64_t ld8,
                  void* __restrict__ codes, float* __restrict__ scale, void* __restrict__ deq,
                  unsigned long long* __restrict__ zero_count) {
     constexpr float qmaxf = static_cast<float>((1 << (BITS - 1)) - 1);
+    const int lane = threadIdx.x & 31;
     const int64_t base = (static_cast<int64_t>(blockIdx.x) * kVecPerThread) * kThreads + threadIdx.x;
     const float2 ones[4] = {make_float2(1.0f, 1.0f), make_float2(1.0f, 1.0f), make_float2(1.0f, 1.0f), make_float2(1.0f, 1.0f)};
+    const bool contiguous = ld8 == C8;
     uint4 w[kVecPerThread];
 #pragma unroll
     for (int k = 0; k < kVecPerThread; ++k) {
         const int64_t idx = base + static_cast<int64_t>(k) * kThreads;
         w[k] = make_uint4(0, 0, 0, 0);
-        if (idx < nvec) w[k] = ld_stream(W + (idx / C8) * ld8 + (idx % C8));
+        if (idx < nvec) w[k] = ld_stream(contiguous ? W + idx : W + (idx / C8) * ld8 + (idx % C8));
+    }
+    // group maxima: the LANES consecutive lanes of a group all end up with it
+    uint32_t m16[kVecPerThread];
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const uint32_t mm = max_u16x2(max_u16x2(w[k].x & 0x7FFF7FFFu, w[k].y & 0x7FFF7FFFu),
+                                      max_u16x2(w[k].z & 0x7FFF7FFFu, w[k].w & 0x7FFF7FFFu));
+        m16[k] = max(mm & 0xFFFFu, mm >> 16);
+#pragma unroll
+        for (int off = LANES / 2; off > 0; off >>= 1) m16[k] = max(m16[k], __shfl_xor_sync(0xFFFFFFFFu, m16[k], off));
+    }
+    // scales d = fl32(max / qmax) and their reciprocals.  A warp holds 32 / LANES groups per vector; with
+    // LANES >= 4 the groups of all its vectors get one lane each, so the warp divides once, not once per vector.
+    float dk[kVecPerThread], rdk[kVecPerThread];
+    if constexpr (LANES >= kVecPerThread) {
+        constexpr int G = 32 / LANES;
+        uint32_t mine = DT == CQ_BF16 ? 0x3F80u : 0x3C00u;        // lanes without a group divide 1.0
+#pragma unroll
+        for (int k = 0; k < kVecPerThread; ++k) {
+            const uint32_t mk = __shfl_sync(0xFFFFFFFFu, m16[k], (lane % G) * LANES);
+            if (lane / G == k) mine = mk;
+        }
+        const float d = __fdiv_rn(cvt16<DT>(static_cast<uint16_t>(mine)), qmaxf);
+        const float rd = guarded_rcp_approx(d);
+#pragma unroll
+        for (int k = 0; k < kVecPerThread; ++k) {
+            dk[k] = __shfl_sync(0xFFFFFFFFu, d, k * G + lane / LANES);
+            rdk[k] = __shfl_sync(0xFFFFFFFFu, rd, k * G + lane / LANES);
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < kVecPerThread; ++k) {
+            dk[k] = __fdiv_rn(cvt16<DT>(static_cast<uint16_t>(m16[k])), qmaxf);
+            rdk[k] = guarded_rcp_approx(dk[k]);
+        }
     }
     unsigned int zeros = 0;
 #pragma unroll
     for (int k = 0; k < kVecPerThread; ++k) {
         const int64_t idx = base + static_cast<int64_t>(k) * kThreads;
-        const uint32_t mm = max_u16x2(max_u16x2(w[k].x & 0x7FFF7FFFu, w[k].y & 0x7FFF7FFFu),
-                                      max_u16x2(w[k].z & 0x7FFF7FFFu, w[k].w & 0x7FFF7FFFu));
-        uint32_t m16 = max(mm & 0xFFFFu, mm >> 16);
-#pragma unroll
-        for (int off = LANES / 2; off > 0; off >>= 1) m16 = max(m16, __shfl_xor_sync(0xFFFFFFFFu, m16, off));
-        const float d = __fdiv_rn(cvt16<DT>(static_cast<uint16_t>(m16)), qmaxf);
-        const float rd = guarded_rcp(d);
+        const float d = dk[k], rd = rdk[k];
         if (idx < nvec) {
             if (scale != nullptr && (idx % LANES) == 0) scale[idx / LANES] = d;
             float2 y2[4], q2[4];

@@ -14,8 +14,15 @@ constexpr int kMaxSmemRowBytes = 221184;   // 216 KB of the 227 KB a CTA may use
 // copy issued by thread 0, so the whole row is in flight at once instead of four vectors per thread.
 __device__ unsigned int g_weight_stage_fault = 0;   // set if the bounded wait on a row copy ever gave up
 
+#ifndef CQ_K4_BULK_MIN_BYTES
+#define CQ_K4_BULK_MIN_BYTES (32 * 1024)
+#endif
+#ifndef CQ_K4_MIN_CTAS
+#define CQ_K4_MIN_CTAS 6
+#endif
+
 template <int DT, int BITS, int DEQ, bool CODES, bool BULK>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, BULK ? 1 : CQ_K4_MIN_CTAS)
 k4_weight_rows(const uint4* __restrict__ W, int C8, int64_t ld8,
                void* __restrict__ codes, float* __restrict__ scale, void* __restrict__ deq,
                unsigned long long* __restrict__ zero_count) {
@@ -70,7 +77,7 @@ k4_weight_rows(const uint4* __restrict__ W, int C8, int64_t ld8,
     for (int v = tid; v < C8; v += kThreads) {
         const uint4 w = s_vec[v];
         float2 y2[4], q2[4];
-        quantize_row8<DT, BITS, true>(w, d, rd, ones, ones, rd == rd, y2, q2);
+        quantize_row8<DT, BITS, true, !BULK>(w, d, rd, ones, ones, rd == rd, y2, q2);
         const int64_t vec = row * C8 + v;
         if constexpr (BITS == 8) {
             const uint32_t c0 = pack_int8x4(y2[0].x, y2[0].y, y2[1].x, y2[1].y);
@@ -241,7 +248,7 @@ static int launch_k4(int64_t R, int C8, int64_t ld8, const void* W, void* codes,
                      unsigned long long* zc, cudaStream_t st) {
     const size_t smem = static_cast<size_t>(C8) * 16;
     // rows of 32 KB or more leave room for at most seven CTAs per SM: those take the bulk-copy variant
-    const bool bulk = smem >= 32 * 1024 && !tuning_no_stage();
+    const bool bulk = smem >= CQ_K4_BULK_MIN_BYTES && !tuning_no_stage();
     auto kern = bulk ? k4_weight_rows<DT, BITS, DEQ, CODES, true> : k4_weight_rows<DT, BITS, DEQ, CODES, false>;
     if (smem > 48 * 1024) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
