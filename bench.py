@@ -42,8 +42,8 @@ HOOK_EVERY = 8
 
 # DRAM traffic of the quantize pass from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum
 # per launch), valid only for the kernel sources whose digest is recorded with it.
-NCU_TRAFFIC = {"sources_sha256": "18648882634bb6549f06a492afa05547557ffa127febf1d8601e8d29f514cef5",
-               "bytes_per_launch": 528703232}   # 235,232,768 read + 293,470,464 written
+NCU_TRAFFIC = {"sources_sha256": "094aa85aae76610fbc303c6995c905582f1e4f05a365b4b1eb8235ee3b23e325",
+               "bytes_per_launch": 527546368}   # 235,186,176 read + 292,360,192 written
 
 
 def kernel_sources_digest() -> str:

@@ -172,12 +172,13 @@ __device__ __forceinline__ float guarded_rcp_approx(float f) {
     asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(f));
     return (f >= kScaleLo && f <= kScaleHi) ? r : __int_as_float(0x7FC00000);
 }
-// The candidate q = round-half-even(v), v = x * (1/a_i) * (1/b_j), is accepted when |v - q| < 1/2 - 2^-12.
+// The candidate q = round-half-even(v), v = x * (1/a_i) * (1/b_j), is accepted when |v - q| < 1/2 - 2^-14.
 // With a_i, b_j in [2^-40, 2^40] they, their reciprocals, s_ij = fl32(a_i b_j) and the reciprocal product
-// are all normal numbers, so v differs from z = x / s_ij by less than 5 * 2^-24 |z| <= 2^-14.6 (|z| <= 128);
-// hence |z - q| < 1/2 - 2^-12 + 2^-14.6 and the IEEE quotient fl32(z), which lies within 2^-17 of z, rounds
-// to the same q.  |x| <= min(t_i, c_j) gives |z| <= qmax (1 + 2^-22), which keeps q within [-qmax, qmax].
-constexpr float kAcceptBelow = 0.499755859375f;         // 1/2 - 2^-12
+// are all normal numbers, so v differs from z = x / s_ij by less than 5 * 2^-24 |z| < 3.8e-5 (five roundings,
+// |z| <= 127.0001); hence |z - q| < 1/2 - 6.1e-5 + 3.8e-5 and the IEEE quotient fl32(z), which lies within
+// 2^-17 = 0.8e-5 of z, stays 1.5e-5 short of the rounding boundary and rounds to the same q.
+// |x| <= min(t_i, c_j) gives |z| <= qmax (1 + 2^-22), which keeps q within [-qmax, qmax].
+constexpr float kAcceptBelow = 0.49993896484375f;       // 1/2 - 2^-14
 
 // Packed fp32x2 arithmetic (bit-identical to the scalar IEEE operations, half the issue slots).
 // y2[k] = kMagic + q and q2[k] = q for elements 2k, 2k+1.  UNIFORM: one scale `a` for the whole row
