@@ -96,6 +96,30 @@ int cq_quantize_act(const void* X, int dtype, int64_t T, int64_t I, int64_t ld,
                     void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * One matrix held in several row blocks (tokens split over GPUs, or X streamed through the device in
+ * chunks): c_j of the CrossQuant equation (Section 4.2) is the maximum over ALL tokens, so the blocks'
+ * column maxima have to be combined before any code is formed; t_i stays local to the block that holds
+ * row i.  These two calls are the per-block steps; what moves the vector between GPUs (an all-reduce
+ * with MAX) is the caller's.
+ *
+ * cq_vector_max: acc_j = max(acc_j, v_j) for j < n, device pointers, in place (acc and v may not overlap
+ * unless equal).  Use it to keep a running c over chunks, or after gathering other blocks' vectors.
+ *
+ * cq_quantize_act_given: cq_quantize_act without its first pass, with t (float[T], this block's rows)
+ * and c (float[I], the combined column maxima) supplied.  Requires t_i >= max_j |X_ij| and
+ * c_j >= max_i |X_ij| for the block (true for maxima combined as above); elements that exceed either
+ * bound get unspecified codes (nothing is checked, nothing faults).  Other arguments, outputs, workspace
+ * and errors as for cq_quantize_act; zero_count counts this block only.
+ */
+int cq_vector_max(float* acc, const float* v, int64_t n, void* stream);
+int cq_quantize_act_given(const void* X, int dtype, int64_t T, int64_t I, int64_t ld,
+                          double alpha, int bits, const float* t, const float* c,
+                          float* row_scale, float* col_scale,
+                          void* codes, void* deq, int deq_dtype,
+                          unsigned long long* zero_count,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * cq_quantize_act for callers that cannot allocate device memory.  (The paper has no counterpart to
  * this function: it exists for deployment, not for the method.)
  *

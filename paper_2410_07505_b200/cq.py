@@ -24,6 +24,7 @@ EXPORTS = (
     "cq_dequantize", "cq_kernel_count", "cq_kernel_count_x", "cq_quantize_weight_per_channel",
     "cq_set_tuning", "cq_set_timing_events", "cq_quantize_act_noalloc",
     "cq_quantize_weight_groupwise", "cq_case_indicators", "cq_remove_kernel", "cq_stage_fault",
+    "cq_vector_max", "cq_quantize_act_given",
 )
 
 
@@ -55,6 +56,9 @@ def lib() -> C.CDLL:
         L.cq_workspace_bytes.argtypes = [i64, i64]
         L.cq_quantize_act.argtypes = [vp, ci, i64, i64, i64, dbl, ci, vp, vp, vp, vp, vp, vp, ci, vp, vp,
                                       C.c_size_t, vp]
+        L.cq_vector_max.argtypes = [vp, vp, i64, vp]
+        L.cq_quantize_act_given.argtypes = [vp, ci, i64, i64, i64, dbl, ci, vp, vp, vp, vp, vp, vp, ci, vp, vp,
+                                            C.c_size_t, vp]
         L.cq_quantize_act_noalloc.argtypes = [vp, ci, i64, i64, i64, dbl, ci, vp, vp, vp, vp, vp, vp, ci, vp, vp]
         L.cq_host_scratch_bytes.restype = C.c_size_t
         L.cq_host_scratch_bytes.argtypes = [i64, i64, ci, ci, ci, ci]
@@ -208,6 +212,35 @@ def quantize_act(X: torch.Tensor, alpha: float = 0.15, bits: int = 8, *, codes: 
 
 
 NOALLOC_SCRATCH_BYTES = 8 << 20
+
+
+def vector_max_(acc: torch.Tensor, v: torch.Tensor) -> torch.Tensor:
+    """acc = max(acc, v) elementwise, in place (float32 device vectors of equal length)."""
+    if acc.dtype != torch.float32 or v.dtype != torch.float32 or acc.numel() != v.numel():
+        raise ValueError("vector_max_ wants two float32 vectors of equal length")
+    _check(lib().cq_vector_max(_ptr(acc), _ptr(v), acc.numel(), _stream()), "cq_vector_max")
+    return acc
+
+
+def quantize_act_given(X: torch.Tensor, t: torch.Tensor, c: torch.Tensor, alpha: float = 0.15, bits: int = 8, *,
+                       codes: bool = True, deq: bool = True, deq_dtype: torch.dtype | None = None, count: bool = True,
+                       buffers: ActBuffers | None = None) -> ActQuant:
+    """CrossQuant of a row block of a larger matrix: t are this block's row maxima, c the column maxima
+    of the whole matrix (combined over all blocks).  The result's t and c are the given vectors."""
+    T, I, ld = _matrix_args(X)
+    if bits == 4 and I % 2:
+        raise CQError(6, "cq_quantize_act_given")
+    if t.dtype != torch.float32 or c.dtype != torch.float32 or t.numel() != T or c.numel() != I:
+        raise ValueError("t must be float32[T] and c float32[I]")
+    b = buffers or ActBuffers(T, I, X.dtype, bits, codes=codes, deq=deq, deq_dtype=deq_dtype, count=count,
+                              device=X.device)
+    deq_dt = _DT[b.deq.dtype] if b.deq is not None else _DT[X.dtype]
+    st = lib().cq_quantize_act_given(_ptr(X), _DT[X.dtype], T, I, ld, float(alpha), int(bits), _ptr(t), _ptr(c),
+                                     _ptr(b.row_scale), _ptr(b.col_scale), _ptr(b.codes), _ptr(b.deq), deq_dt,
+                                     _ptr(b.zero_count), _ptr(b.workspace), b.workspace.numel(), _stream())
+    _check(st, "cq_quantize_act_given")
+    return ActQuant(t=t, c=c, row_scale=b.row_scale, col_scale=b.col_scale, codes=b.codes, deq=b.deq,
+                    zero_count=b.zero_count, bits=bits)
 
 
 def quantize_act_noalloc(X: torch.Tensor, alpha: float = 0.15, bits: int = 8, *, buffers: ActBuffers) -> ActQuant:

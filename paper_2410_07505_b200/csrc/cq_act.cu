@@ -264,6 +264,14 @@ k2_scales_from_vectors(int64_t T, int64_t I, const float* __restrict__ t_in, con
     }
 }
 
+// acc_j = max(acc_j, v_j): combines the maxima of row blocks of one matrix (magnitudes, so never NaN-ordered
+// surprises: fmaxf of two non-negative floats).
+__global__ void __launch_bounds__(kThreads)
+k_vector_max(float* acc, const float* v, int64_t n) {
+    const int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (j < n) acc[j] = fmaxf(acc[j], v[j]);
+}
+
 // ============================================================================ pass 2: quantize
 // Same strip / resident-CTA layout and rolling four-row prefetch as pass 1.  Full row groups are
 // walked from the last one backwards (the rows pass 1 touched last are the likeliest to be still in
@@ -890,6 +898,26 @@ int cq_quantize_act(const void* X, int dtype, int64_t T, int64_t I, int64_t ld, 
                     void* codes, void* deq, int deq_dtype, unsigned long long* zero_count,
                     void* workspace, size_t workspace_bytes, void* stream) {
     return cq::quantize_act_impl(X, dtype, T, I, ld, alpha, bits, nullptr, nullptr, t, c, row_scale, col_scale,
+                                 codes, deq, deq_dtype, zero_count, workspace, workspace_bytes,
+                                 static_cast<cudaStream_t>(stream));
+}
+
+int cq_vector_max(float* acc, const float* v, int64_t n, void* stream) {
+    if (n < 0) return CQ_ERR_SHAPE;
+    if (n == 0) return CQ_OK;
+    if (acc == nullptr || v == nullptr) return CQ_ERR_NULL;
+    if (!cq::aligned(acc, 4) || !cq::aligned(v, 4)) return CQ_ERR_ALIGN;
+    const unsigned blocks = static_cast<unsigned>((n + cq::kThreads - 1) / cq::kThreads);
+    cq::k_vector_max<<<blocks, cq::kThreads, 0, static_cast<cudaStream_t>(stream)>>>(acc, v, n);
+    return cq::launch_status();
+}
+
+int cq_quantize_act_given(const void* X, int dtype, int64_t T, int64_t I, int64_t ld, double alpha, int bits,
+                          const float* t, const float* c, float* row_scale, float* col_scale,
+                          void* codes, void* deq, int deq_dtype, unsigned long long* zero_count,
+                          void* workspace, size_t workspace_bytes, void* stream) {
+    if (T > 0 && I > 0 && (t == nullptr || c == nullptr)) return CQ_ERR_NULL;
+    return cq::quantize_act_impl(X, dtype, T, I, ld, alpha, bits, t, c, nullptr, nullptr, row_scale, col_scale,
                                  codes, deq, deq_dtype, zero_count, workspace, workspace_bytes,
                                  static_cast<cudaStream_t>(stream));
 }

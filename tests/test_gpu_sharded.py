@@ -1,0 +1,99 @@
+"""One matrix in several row blocks (the exchange step of a token-sharded or streamed X): the blocks'
+results, put together, must equal the oracle's on the whole matrix."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import parity
+from paper_2410_07505_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+TORCH_DT = {"f16": torch.float16, "bf16": torch.bfloat16}
+
+
+@pytest.fixture(scope="module")
+def mods():
+    if not torch.cuda.is_available():
+        pytest.fail("the gpu tests need a CUDA device")
+    from paper_2410_07505_b200 import build, cq, sharded
+    build.build()
+    cq.lib()
+    return cq, sharded
+
+
+def to_dev(bits: np.ndarray, dtype: str) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(TORCH_DT[dtype]).cuda()
+
+
+def bits_of(t: torch.Tensor) -> np.ndarray:
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def check_blocks(X, dtype, alpha, bits, outs, total):
+    T, I = X.shape
+    parity.check_act(X, dtype, alpha, bits,
+                     t=np.concatenate([o.t.cpu().numpy() for o in outs]),
+                     c=outs[0].c.cpu().numpy(),
+                     a=np.concatenate([o.row_scale.cpu().numpy() for o in outs]),
+                     b=outs[0].col_scale.cpu().numpy(),
+                     codes=np.concatenate([o.codes.cpu().numpy().reshape(o.t.numel(), -1) for o in outs]),
+                     deq=np.concatenate([bits_of(o.deq).reshape(o.t.numel(), I) for o in outs]),
+                     zero_count=int(total))
+    for o in outs[1:]:                                       # every block used the same column vectors
+        assert torch.equal(o.c, outs[0].c) and torch.equal(o.col_scale, outs[0].col_scale)
+
+
+@pytest.mark.parametrize("shape,cuts", [((301, 1000), (100, 157)), ((64, 2056), (1, 63)), ((50, 77), (20, 21)),
+                                         ((1030, 4104), (512, 1024))])
+@pytest.mark.parametrize("dtype,bits,alpha", [("f16", 8, 0.15), ("bf16", 4, 0.5), ("bf16", 8, 0.0), ("f16", 8, 1.0)])
+def test_row_chunks_equal_the_whole_matrix(mods, shape, cuts, dtype, bits, alpha):
+    cq, sharded = mods
+    T, I = shape
+    if bits == 4 and I % 2:
+        pytest.skip("INT4 packs two columns per byte")
+    X = wl.small_matrix(T, I, dtype, 300 + T + I, outlier_cols=3, zero_frac=0.02)
+    Xd = to_dev(X, dtype)
+    chunks = [Xd[0:cuts[0]], Xd[cuts[0]:cuts[1]], Xd[cuts[1]:T]]
+    outs, total = sharded.quantize_act_chunked(chunks, alpha, bits)
+    torch.cuda.synchronize()
+    check_blocks(X, dtype, alpha, bits, outs, total)
+
+
+def test_running_column_maximum_is_the_column_absmax(mods):
+    cq, _ = mods
+    X = wl.small_matrix(200, 520, "bf16", 5, outlier_cols=4)
+    Xd = to_dev(X, "bf16")
+    _, c_full = cq.absmax_rows_cols(Xd)
+    _, c = cq.absmax_rows_cols(Xd[:70])
+    for r0, r1 in ((70, 71), (71, 200)):
+        cq.vector_max_(c, cq.absmax_rows_cols(Xd[r0:r1])[1])
+    assert torch.equal(c, c_full)
+
+
+def test_row_sharded_call_on_one_rank_equals_the_plain_call(mods):
+    cq, sharded = mods
+    X = wl.small_matrix(130, 2056, "f16", 9, outlier_cols=2, zero_frac=0.01)
+    Xd = to_dev(X, "f16")
+    out, total = sharded.quantize_act_row_sharded(Xd, 0.15, 8)              # no process group: a world of one
+    torch.cuda.synchronize()
+    check_blocks(X, "f16", 0.15, 8, [out], int(total.item()))
+
+
+def test_given_maxima_full_size_sample(mods):
+    """Headline shape in two halves: rows sampled from both halves against the oracle's whole-matrix result."""
+    cq, sharded = mods
+    from oracle import cq_oracle as orc
+    X, cfg = wl.activation("llama70b_attn")
+    Xd = to_dev(X, cfg.dtype)
+    half = cfg.T // 2
+    outs, total = sharded.quantize_act_chunked([Xd[:half], Xd[half:]], 0.15, 8)
+    torch.cuda.synchronize()
+    ref = orc.quantize_act(X, cfg.dtype, 0.15, 8, want_deq16=True)
+    assert total == int(ref.zero_count)
+    rows = np.array([0, 1, half - 1, half, half + 1, cfg.T - 1, 777, 3001])
+    got = np.concatenate([o.codes.cpu().numpy() for o in outs])[rows]
+    assert np.array_equal(got.view(np.int8), ref.codes[rows])
+    assert np.array_equal(outs[0].c.cpu().numpy().view(np.uint32), ref.c.view(np.uint32))

@@ -61,3 +61,52 @@ def test_reference_arm_runs_on_rank_zero_only():
     line = json.loads(p.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["value"] > 0 and line["unit"] == "GB/s"
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
+
+
+# ---- one matrix split by rows over two ranks: the exchange step (column maxima MAX, kernel sizes SUM) ----
+SHARD_WORKER = r"""
+import json, sys
+sys.path.insert(0, {root!r})
+import numpy as np, torch, torch.distributed as dist
+from paper_2410_07505_b200 import sharded, workloads as wl
+dist.init_process_group("gloo", init_method="tcp://127.0.0.1:{port}", rank=int(sys.argv[1]), world_size=2)
+rank = dist.get_rank()
+X = wl.bits_to_f32(wl.small_matrix(37, 24, wl.BF16, 11), wl.BF16)          # the same matrix on both ranks
+r0, r1 = sharded.shard_rows(37, 2, rank)
+c_local = torch.from_numpy(np.abs(X[r0:r1]).max(axis=0).astype(np.float32))    # stands in for the absmax kernel
+c = sharded.combine_column_maxima(c_local.clone())
+total = sharded.combine_counts(torch.tensor(100 + rank, dtype=torch.int64))
+print(json.dumps({{"rank": rank, "rows": [r0, r1], "c": c.tolist(), "c_full": np.abs(X).max(axis=0).tolist(),
+                  "total": int(total)}}))
+dist.barrier()
+dist.destroy_process_group()
+"""
+
+
+def test_row_shards_exchange_column_maxima_and_counts(tmp_path):
+    port = 31500 + os.getpid() % 2000
+    script = tmp_path / "shard_worker.py"
+    script.write_text(SHARD_WORKER.format(root=ROOT, port=port))
+    procs = [subprocess.Popen([sys.executable, str(script), str(r)], stdout=subprocess.PIPE, stderr=subprocess.PIPE,
+                              text=True, cwd=ROOT) for r in range(2)]
+    outs = []
+    for p in procs:
+        out, err = p.communicate(timeout=300)
+        assert p.returncode == 0, err[-2000:]
+        outs.append(json.loads(out.strip().splitlines()[-1]))
+    outs.sort(key=lambda o: o["rank"])
+    assert outs[0]["rows"] == [0, 19] and outs[1]["rows"] == [19, 37]          # contiguous, sizes differ by one
+    for o in outs:
+        assert o["c"] == o["c_full"]                                            # every rank ends with the global maxima
+        assert o["total"] == 201                                                # and with the sum of the counts
+
+
+def test_shard_rows_partition():
+    from paper_2410_07505_b200 import sharded
+    for T in (0, 1, 7, 4096):
+        for world in (1, 2, 3, 8):
+            spans = [sharded.shard_rows(T, world, r) for r in range(world)]
+            assert spans[0][0] == 0 and spans[-1][1] == T
+            assert all(a[1] == b[0] for a, b in zip(spans, spans[1:]))
+            sizes = [b - a for a, b in spans]
+            assert max(sizes) - min(sizes) <= 1
