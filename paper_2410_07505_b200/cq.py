@@ -149,12 +149,21 @@ def absmax_cols(X: torch.Tensor) -> torch.Tensor:
     return c
 
 
-def absmax_rows_cols(X: torch.Tensor):
+def absmax_rows_cols(X: torch.Tensor, *, workspace: torch.Tensor | None = None, out=None):
+    """(t, c) from one read of X.  With a `workspace` (>= workspace_bytes(T, I)) the first pass of
+    cq_quantize_act is used (partial maxima in the workspace, no atomics: faster on large matrices);
+    without one, cq_absmax_rows_cols.  `out` = (t, c) tensors to fill."""
     T, I, ld = _matrix_args(X)
-    t = torch.empty(T, dtype=torch.float32, device=X.device)
-    c = torch.empty(I, dtype=torch.float32, device=X.device)
-    _check(lib().cq_absmax_rows_cols(_ptr(X), _DT[X.dtype], T, I, ld, _ptr(t), _ptr(c), _stream()),
-           "cq_absmax_rows_cols")
+    t, c = out if out is not None else (torch.empty(T, dtype=torch.float32, device=X.device),
+                                        torch.empty(I, dtype=torch.float32, device=X.device))
+    if workspace is None:
+        _check(lib().cq_absmax_rows_cols(_ptr(X), _DT[X.dtype], T, I, ld, _ptr(t), _ptr(c), _stream()),
+               "cq_absmax_rows_cols")
+    else:
+        # alpha = 1 keeps the scale-vector step free of pow; no output but t and c is requested
+        _check(lib().cq_quantize_act(_ptr(X), _DT[X.dtype], T, I, ld, 1.0, 8, _ptr(t), _ptr(c), None, None, None, None,
+                                     _DT[X.dtype], None, _ptr(workspace), workspace.numel(), _stream()),
+               "cq_quantize_act")
     return t, c
 
 

@@ -52,9 +52,11 @@ def quantize_act_row_sharded(X_local: torch.Tensor, alpha: float = 0.15, bits: i
     Returns (ActQuant of the block, with t local and c global; int64 tensor: |K(CQ)| of the whole matrix).
     Identical, block by block, to quantizing the whole matrix on one device.
     """
-    t, c = cq.absmax_rows_cols(X_local)
+    T, I = X_local.shape
+    b = buffers or cq.ActBuffers(T, I, X_local.dtype, bits, device=X_local.device)
+    t, c = cq.absmax_rows_cols(X_local, workspace=b.workspace, out=(b.t, b.c))
     combine_column_maxima(c, group)
-    out = cq.quantize_act_given(X_local, t, c, alpha, bits, buffers=buffers)
+    out = cq.quantize_act_given(X_local, t, c, alpha, bits, buffers=b)
     return out, combine_counts(out.zero_count, group)
 
 
@@ -66,11 +68,11 @@ def quantize_act_chunked(chunks: Sequence[torch.Tensor], alpha: float = 0.15, bi
     """
     if not chunks:
         return [], 0
-    ts, c = [], None
-    for X in chunks:
-        t_k, c_k = cq.absmax_rows_cols(X)
-        ts.append(t_k)
+    bufs = [cq.ActBuffers(X.shape[0], X.shape[1], X.dtype, bits, device=X.device) for X in chunks]
+    c = None
+    for X, b in zip(chunks, bufs):
+        _, c_k = cq.absmax_rows_cols(X, workspace=b.workspace, out=(b.t, b.c))
         c = c_k if c is None else cq.vector_max_(c, c_k)
-    outs = [cq.quantize_act_given(X, t_k, c, alpha, bits) for X, t_k in zip(chunks, ts)]
+    outs = [cq.quantize_act_given(X, b.t, c, alpha, bits, buffers=b) for X, b in zip(chunks, bufs)]
     total = sum(int(o.zero_count.item()) for o in outs)
     return outs, total

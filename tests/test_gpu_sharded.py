@@ -97,3 +97,14 @@ def test_given_maxima_full_size_sample(mods):
     got = np.concatenate([o.codes.cpu().numpy() for o in outs])[rows]
     assert np.array_equal(got.view(np.int8), ref.codes[rows])
     assert np.array_equal(outs[0].c.cpu().numpy().view(np.uint32), ref.c.view(np.uint32))
+
+
+@pytest.mark.parametrize("shape", [(130, 2056), (33, 50), (1, 8)])
+def test_absmax_with_a_workspace_equals_the_atomic_entry_point(mods, shape):
+    cq, _ = mods
+    X = wl.small_matrix(shape[0], shape[1], "bf16", 21, outlier_cols=2, zero_frac=0.05)
+    Xd = to_dev(X, "bf16")
+    ws = torch.empty(cq.workspace_bytes(*shape), dtype=torch.uint8, device="cuda")
+    t0, c0 = cq.absmax_rows_cols(Xd)
+    t1, c1 = cq.absmax_rows_cols(Xd, workspace=ws)
+    assert torch.equal(t0, t1) and torch.equal(c0, c1)
