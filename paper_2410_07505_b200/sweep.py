@@ -74,12 +74,14 @@ def time_extra_ops(Xd: torch.Tensor, alpha: float, flush, iters: int) -> dict:
     us_ind = _time(lambda: cq.case_indicators(r), flush, iters)
     us_cnt = _time(lambda: cq.kernel_count_x(Xd, alpha, 8, t, c, ws), flush, iters)
     us_abs = _time(lambda: cq.absmax_rows_cols(Xd), flush, iters)
+    us_abs_ws = _time(lambda: cq.absmax_rows_cols(Xd, workspace=ws, out=(t, c)), flush, iters)
     _, counts = cq.remove_kernel(Xd, alpha, 8, 1.0, ws)
     ind = cq.case_indicators(r).cpu().tolist()
     cnt = counts.cpu().tolist()
     return {"remove_kernel_us": round(us_rm, 1), "remove_kernel_gbs": round(6 * n / us_rm / 1e3, 1),
             "case_indicators_us": round(us_ind, 1), "kernel_count_x_us": round(us_cnt, 1),
             "absmax_rows_cols_us": round(us_abs, 1), "absmax_gbs": round(2 * n / us_abs / 1e3, 1),
+            "absmax_with_workspace_us": round(us_abs_ws, 1),
             "kernel_proportion_per_token": cnt[1] / n, "kernel_proportion_crossquant": cnt[2] / n,
             "share_c_ge_t": ind[0] / n, "share_bound_smaller": ind[1] / n}
 
