@@ -91,11 +91,16 @@ def main() -> None:
     ap.add_argument("--iters", type=int, default=30)
     ap.add_argument("--layers", type=int, default=0, help="layers of the 80-layer sweep to run (0 = skip)")
     ap.add_argument("--alpha", type=float, default=0.15)
+    ap.add_argument("--only", default="", help="comma-separated config names (e.g. llama70b_mlp,weight_8192x28672): "
+                    "time only these (keeps a profiler capture short)")
     args = ap.parse_args()
+    only = set(filter(None, args.only.split(",")))
     cq.lib()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
 
     for name, cfg in wl.ACT_CONFIGS.items():
+        if only and name not in only:
+            continue
         Xd = _dev(wl.generate_activation(cfg), cfg.dtype)
         for bits in cfg.bits:
             for alpha in cfg.alphas:
@@ -108,6 +113,8 @@ def main() -> None:
             print(json.dumps(row), flush=True)
         del Xd
     for k, shape in enumerate(wl.SWEEP_WEIGHT_SHAPES):
+        if only and f"weight_{shape[0]}x{shape[1]}" not in only:
+            continue
         Wd = _dev(wl.sweep_weight(0, k), "bf16")
         for bits in (8, 4):
             row = {"config": f"weight_{shape[0]}x{shape[1]}", "shape": list(shape), "dtype": "bf16", "bits": bits}
