@@ -278,6 +278,32 @@ def test_weight_groupwise(cq, shape, group, bits):
         parity.check_weight(W, dtype, bits, deq=r.deq.cpu().numpy(), deq_is_f32=True, ref=ref)
 
 
+@pytest.mark.parametrize("bits,top", [(8, 254), (4, 14)])
+def test_rows_full_of_exact_ties(cq, bits, top):
+    """A row maximum of 2 * qmax * 2^e puts every odd multiple of 2^e on a rounding tie (x / d = k / 2): the
+    re-examination path has to settle them all to the even neighbour, for weights, groups and activations."""
+    rng = np.random.Generator(np.random.PCG64(77))
+    for dtype in ("bf16", "f16"):
+        for e in (-10, 0, 3):
+            k = rng.integers(-top, top + 1, size=(37, 1024)).astype(np.float32)
+            k[:, ::128] = top                                  # every group of 128 holds the maximum
+            k[5, :] = 0
+            W = wl.to_bits(k * np.float32(2.0 ** e), dtype)
+            assert np.array_equal(wl.bits_to_f32(W, dtype), k * np.float32(2.0 ** e))   # exactly representable
+            Wd = to_dev(W, dtype)
+            ref = orc.quantize_weight_per_channel(W, dtype, bits)
+            r = cq.quantize_weight_per_channel(Wd, bits)
+            parity.check_weight(W, dtype, bits, scale=r.scale.cpu().numpy(), codes=r.codes.cpu().numpy(),
+                                deq=bits_of(r.deq), zero_count=int(r.zero_count.item()), ref=ref)
+            refg = orc.quantize_weight_groupwise(W, dtype, bits, 128)
+            g = cq.quantize_weight_groupwise(Wd, 128, bits)
+            parity.check_weight(W, dtype, bits, scale=g.scale.cpu().numpy(), codes=g.codes.cpu().numpy(),
+                                deq=bits_of(g.deq), zero_count=int(g.zero_count.item()), ref=refg)
+            run_and_check(cq, W, dtype, 1.0, bits, Xd=Wd)      # per-token activations: the same ties
+            ties = np.abs(k / 2 - np.trunc(k / 2)) == 0.5
+            assert ties.mean() > 0.3
+
+
 def test_weight_groupwise_rejects_a_group_that_does_not_divide_the_row(cq):
     Wd = torch.zeros((4, 100), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(cq.CQError) as e:
@@ -298,6 +324,40 @@ def test_remove_kernel(cq, shape, dtype):
         torch.cuda.synchronize()
         assert counts.cpu().tolist() == [removed, k_pt, k_cq]
         assert np.array_equal(bits_of(out), want)
+
+
+def test_zero_tests_on_exact_boundaries_and_extreme_scales(cq):
+    """The diagnostics kernel decides |fl32(x/s)| <= h from products and thresholds; the cases it must hand
+    to the quotient: elements exactly on the bound, neighbours of the bound, scales and bounds outside
+    the range the shortcut covers."""
+    # per-token rows with s_i = 2^k: x = s/2 is exactly on the bound 1/2 (code 0 by round-half-even)
+    rows = []
+    for k in (-6, 0, 5):
+        s = np.float32(2.0 ** k)
+        r = np.zeros(264, dtype=np.float32)
+        r[0] = 127 * s                                     # row maximum: the scale is exactly s
+        r[1:9] = np.array([0.5, -0.5, 1.5, 2.5, 0.49609375, 0.50390625, 0.25, 0.75], dtype=np.float32) * s
+        r[9:] = np.linspace(-3, 3, 255, dtype=np.float32) * s
+        rows.append(r)
+    for dtype in ("f16", "bf16"):
+        X = wl.to_bits(np.stack(rows * 3), dtype)
+        Xd = to_dev(X, dtype)
+        for alpha, theta in [(1.0, 1.0), (1.0, 3.0), (0.0, 1.0), (0.3, 1.0), (1.0, 1e-30), (1.0, 1e30), (0.5, 2.0 ** -21)]:
+            want, removed, k_pt, k_cq = orc.remove_kernel(X, dtype, alpha, 8, theta)
+            out, counts = cq.remove_kernel(Xd, alpha, 8, theta)
+            assert counts.cpu().tolist() == [removed, k_pt, k_cq], (dtype, alpha, theta)
+            assert np.array_equal(bits_of(out), want)
+            t, c = cq.absmax_rows_cols(Xd)
+            assert int(cq.kernel_count_x(Xd, alpha, 8, t, c).item()) == k_cq
+    # scale factors outside [2^-40, 2^40]: everything goes through the quotient
+    for scale in (1e36, 1e-36, 3e-39):
+        B = wl.small_matrix(24, 128, "bf16", 4, scale=scale, outlier_cols=1, outlier_scale=8.0, zero_frac=0.05)
+        Bd = to_dev(B, "bf16")
+        for alpha in (0.0, 0.15, 1.0):
+            want, removed, k_pt, k_cq = orc.remove_kernel(B, "bf16", alpha, 8, 1.0)
+            out, counts = cq.remove_kernel(Bd, alpha, 8, 1.0)
+            assert counts.cpu().tolist() == [removed, k_pt, k_cq], (scale, alpha)
+            assert np.array_equal(bits_of(out), want)
 
 
 @pytest.mark.parametrize("shape", [(48, 80), (300, 1536), (65, 7), (1, 1)])
