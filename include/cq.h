@@ -234,11 +234,14 @@ int cq_remove_kernel(const void* X, int dtype, int64_t T, int64_t I, int64_t ld,
 int cq_case_indicators(const float* t, const float* c, const float* row_scale, const float* col_scale,
                        int64_t T, int64_t I, int bits, unsigned long long* counts, void* stream);
 
-/* Launch-shape knobs for measurement.  key: "k1_ctas_per_sm", "k3_ctas_per_sm" (resident CTAs per SM
- * the two passes size their grids for; 1..64; for the staged quantize pass 2 or 3 picks the build for that occupancy), "k3_forward" (1: the quantize pass walks the rows in
- * ascending order) or "no_pdl" (1: launch the quantize pass without programmatic dependent launch), "no_stage" (1: the quantize pass
- * loads rows straight into registers instead of staging them in shared memory with bulk copies).  value <= 0 restores the built-in choice.  Results never depend on these.
- * Returns CQ_OK or CQ_ERR_SHAPE. */
+/* Launch-shape knobs for measurement.  Results never depend on them.  key:
+ *   "k1_ctas_per_sm", "k3_ctas_per_sm"  resident CTAs per SM the two passes size their grids for (1..64); for the
+ *                                       staged quantize pass 2 or 3 picks the build for that occupancy
+ *   "k3_forward"  1: the quantize pass walks the rows in ascending order
+ *   "no_pdl"      1: no programmatic dependent launch (quantize pass and diagnostics passes)
+ *   "no_stage"    1: the quantize pass loads rows straight into registers instead of staging them in shared memory
+ *                    with bulk copies; the weight quantizer uses plain loads for long rows too
+ * value <= 0 restores the built-in choice.  Returns CQ_OK or CQ_ERR_SHAPE (unknown key). */
 int cq_set_tuning(const char* key, int value);
 
 /* Health check.  The quantize pass, the diagnostics passes (cq_remove_kernel, cq_kernel_count_x) and the
