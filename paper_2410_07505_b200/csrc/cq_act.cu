@@ -556,17 +556,20 @@ static bool fast_input(const void* X, int64_t I, int64_t ld) {
 int launch_status() { return cudaGetLastError() == cudaSuccess ? CQ_OK : CQ_ERR_CUDA; }
 
 int sm_count() {
+    static int known[64] = {};                       // per device; 0 = not asked yet (a benign race: same value)
     int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-        n = 148;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (dev >= 0 && dev < 64 && known[dev] > 0) return known[dev];
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+    if (dev >= 0 && dev < 64) known[dev] = n;
     return n;
 }
 
 // CTAs per column strip so that the whole grid is resident at once: floor(SMs * CTAs/SM / strips).
 template <typename Kernel>
-static int resident_y(Kernel kern, int W, int nstrips, int64_t ngroups, int tuned_ctas_per_sm, int cap) {
+static int resident_y(Kernel kern, int W, int nstrips, int64_t ngroups, int tuned_ctas_per_sm, int cap, LaunchMemo& memo) {
     int per_sm = tuned_ctas_per_sm;
-    if (per_sm <= 0 && cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, W, 0) != cudaSuccess) per_sm = 1;
+    if (per_sm <= 0) per_sm = resident_ctas(kern, W, 0, 0, memo);
     if (per_sm < 1) per_sm = 1;
     int64_t y = static_cast<int64_t>(sm_count()) * per_sm / nstrips;
     if (y > ngroups) y = ngroups;
@@ -580,7 +583,8 @@ template <bool ATOMIC, int DT>
 static int launch_k1(const Plan& p, const void* X, int64_t T, int64_t ld, uint16_t* rowpart, uint16_t* colpart,
                      float* t, float* c, cudaStream_t st) {
     auto kern = k1_absmax<ATOMIC, DT>;
-    const int Y = resident_y(kern, p.W, p.nstrips, (p.ngroups * 4 + kG1 - 1) / kG1, g_tune_k1_ctas, ATOMIC ? 0 : p.ycap);
+    static thread_local LaunchMemo memo;
+    const int Y = resident_y(kern, p.W, p.nstrips, (p.ngroups * 4 + kG1 - 1) / kG1, g_tune_k1_ctas, ATOMIC ? 0 : p.ycap, memo);
     kern<<<dim3(p.nstrips, Y), p.W, 0, st>>>(static_cast<const uint4*>(X), T, p.I8, ld / 8, p.nstrips, rowpart,
                                              reinterpret_cast<uint4*>(colpart), t, c);
     return Y;
@@ -634,12 +638,9 @@ template <int DT, int BITS, int DEQ, bool CODES, bool COUNT, int MODE>
 static bool launch_k3_staged(const Plan& p, const K3Args& k, cudaStream_t st) {
     auto kern = k3_quantize<DT, BITS, DEQ, CODES, COUNT, MODE>;
     const size_t smem = static_cast<size_t>(kStages) * 4 * p.W * 16;
-    int per_sm = 0;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, p.W, smem) != cudaSuccess || per_sm < 1) {
-        cudaGetLastError();
-        return false;
-    }
+    static thread_local LaunchMemo memo;
+    const int per_sm = resident_ctas(kern, p.W, smem, static_cast<size_t>(kStages) * 4 * kThreads * 16, memo);
+    if (per_sm < 1) return false;
     int64_t y = static_cast<int64_t>(sm_count()) * per_sm / p.nstrips;
     if (y > p.ngroups) y = p.ngroups;
     if (y > 65535) y = 65535;
@@ -661,7 +662,8 @@ static void launch_k3_one(const Plan& p, const K3Args& k, cudaStream_t st) {
         if (ok) return;
     }
     auto kern = k3_quantize<DT, BITS, DEQ, CODES, COUNT, 0>;
-    const int Y = resident_y(kern, p.W, p.nstrips, p.ngroups, g_tune_k3_ctas, 0);
+    static thread_local LaunchMemo memo;
+    const int Y = resident_y(kern, p.W, p.nstrips, p.ngroups, g_tune_k3_ctas, 0, memo);
     launch_dependent(kern, dim3(p.nstrips, Y), dim3(p.W), 0, st, k.X, k.T, k.I8, k.ld8, k.a, k.ra, k.b, k.rb, k.codes,
                      k.deq, k.zc, g_tune_k3_forward);
 }

@@ -321,12 +321,9 @@ template <int DT, bool WRITE, bool DUAL, bool SAME>
 static bool launch_k9(const Plan& p, const ZeroArgs& z, cudaStream_t st) {
     auto kern = k9_zero_tests<DT, WRITE, DUAL, SAME>;
     const size_t smem = static_cast<size_t>(kRing) * 4 * p.W * 16;
-    int per_sm = 0;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, p.W, smem) != cudaSuccess || per_sm < 1) {
-        cudaGetLastError();
-        return false;
-    }
+    static thread_local LaunchMemo memo;
+    const int per_sm = resident_ctas(kern, p.W, smem, static_cast<size_t>(kRing) * 4 * kThreads * 16, memo);
+    if (per_sm < 1) return false;
     int64_t y = static_cast<int64_t>(sm_count()) * per_sm / p.nstrips;
     if (y > p.ngroups) y = p.ngroups;
     if (y > 65535) y = 65535;

@@ -34,4 +34,29 @@ int weight_stage_fault(unsigned int* fault_host); // flag of the bulk-copy weigh
 bool tuning_no_stage();   // staged (bulk-copy) variants switched off through cq_set_tuning
 bool tuning_no_pdl();     // programmatic dependent launch switched off through cq_set_tuning
 
+// What the runtime answered for one kernel at (device, block size, dynamic shared memory): resident CTAs
+// per SM, after raising the kernel's dynamic shared-memory limit to `smem_limit` (the most any launch of
+// that kernel asks for, so the limit never shrinks whatever the order of shapes and threads).
+// One memo per launch site (a thread_local static there), so repeated calls of one shape ask only once.
+struct LaunchMemo { int dev = -1; int block = 0; size_t smem = 0; int per_sm = 0; };
+
+template <typename Kernel>
+inline int resident_ctas(Kernel kern, int block, size_t smem, size_t smem_limit, LaunchMemo& memo) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (memo.dev == dev && memo.block == block && memo.smem == smem) return memo.per_sm;
+    int per_sm = 0;
+    if (smem_limit > 48 * 1024 &&
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_limit)) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, block, smem) != cudaSuccess || per_sm < 1) {
+        cudaGetLastError();
+        return 0;
+    }
+    memo = LaunchMemo{dev, block, smem, per_sm};
+    return per_sm;
+}
+
 }  // namespace cq

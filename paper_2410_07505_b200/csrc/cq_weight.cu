@@ -250,10 +250,8 @@ static int launch_k4(int64_t R, int C8, int64_t ld8, const void* W, void* codes,
     // rows of 32 KB or more leave room for at most seven CTAs per SM: those take the bulk-copy variant
     const bool bulk = smem >= CQ_K4_BULK_MIN_BYTES && !tuning_no_stage();
     auto kern = bulk ? k4_weight_rows<DT, BITS, DEQ, CODES, true> : k4_weight_rows<DT, BITS, DEQ, CODES, false>;
-    if (smem > 48 * 1024) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
-            return CQ_ERR_CUDA;
-    }
+    static thread_local LaunchMemo memo[2];          // raises the dynamic shared-memory limit once per row length
+    if (smem > 48 * 1024 && resident_ctas(kern, kThreads, smem, kMaxSmemRowBytes, memo[bulk ? 1 : 0]) < 1) return CQ_ERR_CUDA;
     kern<<<static_cast<unsigned>(R), kThreads, smem, st>>>(static_cast<const uint4*>(W), C8, ld8, codes, scale, deq, zc);
     return launch_status();
 }
