@@ -60,6 +60,33 @@ def quantize_act_row_sharded(X_local: torch.Tensor, alpha: float = 0.15, bits: i
     return out, combine_counts(out.zero_count, group)
 
 
+def quantize_act_col_sharded(X_local: torch.Tensor, alpha: float = 0.15, bits: int = 8, *, group=None,
+                             buffers: "cq.ActBuffers | None" = None):
+    """The same for channels split over the ranks (how tensor-parallel FC2 inputs arrive): the column maxima
+    are local, the row maxima t_i are combined (all-reduce MAX of T floats).  X_local may be a column slice
+    of a wider matrix (rows `stride(0)` apart).  Returns (ActQuant with t global and c local, total count)."""
+    T, I = X_local.shape
+    b = buffers or cq.ActBuffers(T, I, X_local.dtype, bits, device=X_local.device)
+    t, c = cq.absmax_rows_cols(X_local, workspace=b.workspace, out=(b.t, b.c))
+    combine_column_maxima(t, group)            # the same exchange, on the other vector
+    out = cq.quantize_act_given(X_local, t, c, alpha, bits, buffers=b)
+    return out, combine_counts(out.zero_count, group)
+
+
+def quantize_act_column_blocks(blocks: Sequence[torch.Tensor], alpha: float = 0.15, bits: int = 8):
+    """One device, the matrix given as column blocks (each [T, I_k], same T): running maximum of t over the
+    blocks, then each block quantized with the final t and its own c.  Returns (list of ActQuant, total)."""
+    if not blocks:
+        return [], 0
+    bufs = [cq.ActBuffers(X.shape[0], X.shape[1], X.dtype, bits, device=X.device) for X in blocks]
+    t = None
+    for X, b in zip(blocks, bufs):
+        t_k, _ = cq.absmax_rows_cols(X, workspace=b.workspace, out=(b.t, b.c))
+        t = t_k if t is None else cq.vector_max_(t, t_k)
+    outs = [cq.quantize_act_given(X, t, b.c, alpha, bits, buffers=b) for X, b in zip(blocks, bufs)]
+    return outs, sum(int(o.zero_count.item()) for o in outs)
+
+
 def quantize_act_chunked(chunks: Sequence[torch.Tensor], alpha: float = 0.15, bits: int = 8):
     """CrossQuant of a matrix that passes through the device as row chunks (each [T_k, I], same I).
 

@@ -108,3 +108,28 @@ def test_absmax_with_a_workspace_equals_the_atomic_entry_point(mods, shape):
     t0, c0 = cq.absmax_rows_cols(Xd)
     t1, c1 = cq.absmax_rows_cols(Xd, workspace=ws)
     assert torch.equal(t0, t1) and torch.equal(c0, c1)
+
+
+@pytest.mark.parametrize("shape,cuts", [((130, 2056), (1024, 1544)), ((64, 4104), (8, 2056)), ((37, 90), (30, 31))])
+@pytest.mark.parametrize("dtype,bits,alpha", [("bf16", 8, 0.15), ("f16", 4, 0.5), ("bf16", 8, 1.0)])
+def test_column_blocks_equal_the_whole_matrix(mods, shape, cuts, dtype, bits, alpha):
+    cq, sharded = mods
+    T, I = shape
+    if bits == 4 and any(c % 2 for c in cuts):
+        pytest.skip("INT4 packs two columns per byte")
+    X = wl.small_matrix(T, I, dtype, 500 + T + I, outlier_cols=3, zero_frac=0.02)
+    Xd = to_dev(X, dtype)
+    blocks = [Xd[:, 0:cuts[0]], Xd[:, cuts[0]:cuts[1]], Xd[:, cuts[1]:I]]        # views: rows I elements apart
+    outs, total = sharded.quantize_act_column_blocks(blocks, alpha, bits)
+    torch.cuda.synchronize()
+    from oracle import cq_oracle as orc
+    ref = orc.quantize_act(X, dtype, alpha, bits, want_deq32=False, want_deq16=True)
+    assert total == int(ref.zero_count)
+    edges = [0, cuts[0], cuts[1], I]
+    for o, j0, j1 in zip(outs, edges[:-1], edges[1:]):
+        assert np.array_equal(o.t.cpu().numpy().view(np.uint32), ref.t.view(np.uint32))
+        assert np.array_equal(o.c.cpu().numpy().view(np.uint32), ref.c[j0:j1].view(np.uint32))
+        codes = o.codes.cpu().numpy()
+        codes = parity.unpack_int4(codes, T, j1 - j0) if bits == 4 else codes.view(np.int8)
+        assert np.array_equal(codes, ref.codes[:, j0:j1])
+        assert np.array_equal(bits_of(o.deq).reshape(T, j1 - j0), ref.deq16[:, j0:j1])
