@@ -3,9 +3,10 @@
 // Pass 1 reads X once and produces partial row maxima (one per row and column strip) and partial
 // column maxima (one per column and resident CTA) of the 15-bit magnitudes; a small second kernel
 // finishes both reductions and writes t, c and the scale vectors, so no atomics or zero-initialised
-// buffers are involved and the result does not depend on scheduling.  Pass 2 re-reads X (walking the rows in the opposite order; the rows
-// arrive through a shared-memory ring filled by asynchronous bulk copies), forms s_ij = a_i * b_j in
-// registers and emits codes, the dequantized matrix and the number of zero codes.
+// buffers are involved and the result does not depend on scheduling.  Pass 2 re-reads X (walking the
+// rows in the opposite order; the rows arrive through a shared-memory ring filled by asynchronous bulk
+// copies), forms s_ij = a_i * b_j in registers and emits codes, the dequantized matrix and the number
+// of zero codes.
 #include <math.h>
 
 #include <initializer_list>

@@ -19,7 +19,6 @@ constexpr float kHalfMinus = 0.4999847412109375f;
 
 constexpr float kScaleLoTie = 2.350988701644575e-38f;    // 2^-125: s / 2 is a normal number, hence exact, from here up
 constexpr int kThreads = 256;      // largest CTA of the tiled kernels
-constexpr int kMaxRowsPerCta = 128;
 
 __device__ __forceinline__ uint32_t max_u16x2(uint32_t a, uint32_t b) {
     uint32_t r;

@@ -312,7 +312,7 @@ static void launch_after(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t s
 
 struct ZeroArgs {
     const void* X; int64_t T; int64_t I; int64_t ld;
-    const float *t, *a, *ra, *b, *rb;
+    const float *t, *a, *b, *rb;
     float qmaxf, half_bound;
     void* out; unsigned long long* counts;
 };
@@ -356,8 +356,8 @@ static ZeroArgs zero_args(const Plan& p, void* workspace, const void* X, int64_t
                           int bits, float half_bound, void* out, unsigned long long* counts) {
     char* ws = static_cast<char*>(workspace);
     return ZeroArgs{X, T, I, ld, t,
-                    reinterpret_cast<const float*>(ws + p.off_a), reinterpret_cast<const float*>(ws + p.off_ra),
-                    reinterpret_cast<const float*>(ws + p.off_b), reinterpret_cast<const float*>(ws + p.off_rb),
+                    reinterpret_cast<const float*>(ws + p.off_a), reinterpret_cast<const float*>(ws + p.off_b),
+                    reinterpret_cast<const float*>(ws + p.off_rb),
                     static_cast<float>((1 << (bits - 1)) - 1), half_bound, out, counts};
 }
 
