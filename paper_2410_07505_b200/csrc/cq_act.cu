@@ -23,24 +23,6 @@
 
 namespace cq {
 
-// ============================================================================ scale factors
-//   a_i = fl32(pow(t_i, alpha) / qmax), b_j = fl32(pow(c_j, 1 - alpha)) in fp64, with alpha in {0, 1}
-//   special-cased so that they reduce exactly to per-column / per-token quantization, plus the
-//   reciprocals the quantize pass uses for its candidate codes.
-__device__ __forceinline__ void row_scale_of(float ti, double alpha, int qmax, float& ai, float& rai) {
-    if (alpha == 1.0) ai = __fdiv_rn(ti, static_cast<float>(qmax));
-    else if (alpha == 0.0) ai = 1.0f;
-    else ai = static_cast<float>(pow(static_cast<double>(ti), alpha) / static_cast<double>(qmax));
-    rai = guarded_rcp(ai);
-}
-
-__device__ __forceinline__ void col_scale_of(float cj, double alpha, int qmax, float& bj, float& rbj) {
-    if (alpha == 1.0) bj = 1.0f;
-    else if (alpha == 0.0) bj = __fdiv_rn(cj, static_cast<float>(qmax));
-    else bj = static_cast<float>(pow(static_cast<double>(cj), 1.0 - alpha));
-    rbj = guarded_rcp(bj);
-}
-
 // ============================================================================ pass 1: absmax
 // Grid: x = column strip (blockDim.x vectors of 8 columns), y = one of Y resident CTAs per strip.
 // CTA y walks the row groups (kG1 rows each) y, y+Y, y+2Y, ...  Each of its row slots is re-loaded
@@ -493,6 +475,7 @@ static int g_tune_k1_ctas = 0;      // resident CTAs per SM assumed for pass 1 (
 static int g_tune_k3_ctas = 0;      // the same for pass 2
 static int g_tune_k3_forward = 0;   // walk pass 2 in ascending row order
 static int g_tune_no_pdl = 0;       // launch pass 2 without programmatic dependent launch
+static int g_tune_no_small = 0;     // never take the single-launch path for small matrices
 static int g_tune_no_stage = 0;     // pass 2 loads rows straight into registers instead of staging them
 static cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
 
@@ -751,6 +734,20 @@ int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
                           T * static_cast<int64_t>(p.I8) < (int64_t(1) << 31);     // 32-bit vector indices
     const unsigned k2v_blocks = static_cast<unsigned>((T + I + kThreads - 1) / kThreads);
 
+    // ---- small matrices: everything in one launch of one thread-block cluster
+    if (!given && fast_in && fast_out && !g_tune_no_small && (g_ev_before == nullptr || g_ev_after == nullptr) &&
+        (codes != nullptr || deq != nullptr || zero_count != nullptr)) {      // (callers without outputs want the workspace vectors)
+        const SmallArgs sa{X, dtype, T, p.I8, ld / 8, p.W, p.nstrips, alpha, bits, t_dev, c_dev, a_dev, b_dev,
+                           codes, deq, deq == nullptr ? 0 : (deq_dtype == CQ_F32 ? 2 : 1), zero_count};
+        if (launch_small(sa, st)) {
+            if ((rc = launch_status()) != CQ_OK) return rc;
+            if (col_scale != nullptr && !b_in_place &&
+                cudaMemcpyAsync(col_scale, b_dev, sizeof(float) * I, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+                return CQ_ERR_CUDA;
+            return CQ_OK;
+        }
+    }
+
     // ---- pass 1 + scale vectors
     if (given) {
         k2_scales_from_vectors<<<k2v_blocks, kThreads, 0, st>>>(T, I, t_given, c_given, alpha, qmax, a_dev, b_dev,
@@ -850,17 +847,19 @@ int cq_set_tuning(const char* key, int value) {
     if (eq(key, "k3_forward")) { cq::g_tune_k3_forward = v ? 1 : 0; return CQ_OK; }
     if (eq(key, "no_pdl")) { cq::g_tune_no_pdl = v ? 1 : 0; return CQ_OK; }
     if (eq(key, "no_stage")) { cq::g_tune_no_stage = v ? 1 : 0; return CQ_OK; }
+    if (eq(key, "no_small")) { cq::g_tune_no_small = v ? 1 : 0; return CQ_OK; }
     return CQ_ERR_SHAPE;
 }
 
 int cq_stage_fault(unsigned int* fault_host) {
     if (fault_host == nullptr) return CQ_ERR_NULL;
-    unsigned int quantize_pass = 0, diagnostics = 0, weights = 0;
+    unsigned int quantize_pass = 0, diagnostics = 0, weights = 0, small = 0;
     if (cudaMemcpyFromSymbol(&quantize_pass, cq::g_stage_fault, sizeof(unsigned int)) != cudaSuccess) return CQ_ERR_CUDA;
     int rc = cq::diag_stage_fault(&diagnostics);
     if (rc == CQ_OK) rc = cq::weight_stage_fault(&weights);
+    if (rc == CQ_OK) rc = cq::small_stage_fault(&small);
     if (rc != CQ_OK) return rc;
-    *fault_host = quantize_pass | diagnostics | weights;
+    *fault_host = quantize_pass | diagnostics | weights | small;
     return CQ_OK;
 }
 

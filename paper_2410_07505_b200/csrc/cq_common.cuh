@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
+#include <math.h>
 #include <stdint.h>
 
 #include "cq.h"
@@ -171,6 +172,24 @@ __device__ __forceinline__ float guarded_rcp_approx(float f) {
     asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(f));
     return (f >= kScaleLo && f <= kScaleHi) ? r : __int_as_float(0x7FC00000);
 }
+// ---- scale factors -------------------------------------------------------------------------
+//   a_i = fl32(pow(t_i, alpha) / qmax), b_j = fl32(pow(c_j, 1 - alpha)) in fp64, with alpha in {0, 1}
+//   special-cased so that they reduce exactly to per-column / per-token quantization, plus the
+//   reciprocals the quantize pass uses for its candidate codes.
+__device__ __forceinline__ void row_scale_of(float ti, double alpha, int qmax, float& ai, float& rai) {
+    if (alpha == 1.0) ai = __fdiv_rn(ti, static_cast<float>(qmax));
+    else if (alpha == 0.0) ai = 1.0f;
+    else ai = static_cast<float>(pow(static_cast<double>(ti), alpha) / static_cast<double>(qmax));
+    rai = guarded_rcp(ai);
+}
+
+__device__ __forceinline__ void col_scale_of(float cj, double alpha, int qmax, float& bj, float& rbj) {
+    if (alpha == 1.0) bj = 1.0f;
+    else if (alpha == 0.0) bj = __fdiv_rn(cj, static_cast<float>(qmax));
+    else bj = static_cast<float>(pow(static_cast<double>(cj), 1.0 - alpha));
+    rbj = guarded_rcp(bj);
+}
+
 // The candidate q = round-half-even(v), v = x * (1/a_i) * (1/b_j), is accepted when |v - q| < 1/2 - 2^-14.
 // With a_i, b_j in [2^-40, 2^40] they, their reciprocals, s_ij = fl32(a_i b_j) and the reciprocal product
 // are all normal numbers, so v differs from z = x / s_ij by less than 5 * 2^-24 |z| < 3.8e-5 (five roundings,

@@ -25,6 +25,16 @@ int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
                       void* codes, void* deq, int deq_dtype, unsigned long long* zero_count,
                       void* workspace, size_t ws_bytes, cudaStream_t st);
 
+// The single-launch path for small matrices (cq_small.cu).  Returns false, having launched nothing, when
+// the shape is not eligible.  All pointers except codes / deq / zero_count are non-null device pointers.
+struct SmallArgs {
+    const void* X; int dtype; int64_t T; int I8; int64_t ld8; int W; int nstrips; double alpha; int bits;
+    float *t, *c, *a, *b;
+    void* codes; void* deq; int deq_mode; unsigned long long* zero_count;
+};
+bool launch_small(const SmallArgs& s, cudaStream_t st);
+int small_stage_fault(unsigned int* fault_host);   // flag of its tile copy
+
 int scales_from_vectors(int64_t T, int64_t I, const float* t, const float* c, double alpha, int bits,
                         void* workspace, size_t ws_bytes, unsigned long long* to_zero, cudaStream_t st);
 int sm_count();

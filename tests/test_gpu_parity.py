@@ -162,6 +162,34 @@ def test_tiling_knobs_do_not_change_results(cq):
             cq.set_tuning(key, 0)
 
 
+SMALL_SHAPES = [(1, 8), (1, 4096), (3, 16), (16, 4096), (16, 8192), (32, 2048), (31, 776), (9, 5000), (5, 8200), (16, 6152),
+                (33, 2048), (17, 8192)]
+
+
+@pytest.mark.parametrize("shape", SMALL_SHAPES)
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+def test_small_matrices_one_launch_and_three_launches(cq, shape, dtype):
+    """Decode-sized matrices take a single thread-block-cluster launch (up to 4 rows per cluster CTA, up to four
+    column strips); the shapes around its limits and the same shapes forced through the three launches."""
+    T, I = shape
+    X = wl.small_matrix(T, I, dtype, 700 + T + I, outlier_cols=3, outlier_scale=30.0, zero_frac=0.03)
+    X[0, : min(I, 24)] = 0
+    Xd = to_dev(X, dtype)
+    try:
+        for no_small in (0, 1):
+            cq.set_tuning("no_small", no_small)
+            for alpha, bits in [(0.15, 8), (0.5, 4), (1.0, 8), (0.0, 4)]:
+                if bits == 4 and I % 2:
+                    continue
+                run_and_check(cq, X, dtype, alpha, bits, Xd=Xd)
+            run_and_check(cq, X, dtype, 0.15, 8, deq_f32=True, Xd=Xd)
+            r = cq.quantize_act(Xd, 0.15, 8, codes=False, deq=False)          # count only
+            assert int(r.zero_count.item()) == orc.quantize_act(X, dtype, 0.15, 8, want_deq32=False, want_deq16=False).zero_count
+    finally:
+        cq.set_tuning("no_small", 0)
+    assert cq.stage_fault() == 0
+
+
 def test_launch_without_programmatic_dependent_launch_gives_the_same_results(cq):
     try:
         cq.set_tuning("no_pdl", 1)
