@@ -76,7 +76,8 @@ size_t cq_workspace_bytes(int64_t T, int64_t I);
 
 /*
  * The CrossQuant activation quantizer (Section 4.2): absmax vectors, scale vectors, codes,
- * dequantized matrix and the size of the quantization kernel (Definition 1), in three launches.
+ * dequantized matrix and the size of the quantization kernel (Definition 1), in three launches
+ * (decode-sized matrices: one launch of one thread-block cluster, same results).
  *   X          in   device [T x ld], dtype CQ_F16 or CQ_BF16
  *   alpha      in   exponent of the row maxima, [0, 1]; 1 = per-token (Eq. 1), 0 = per-column
  *   bits       in   8 or 4
@@ -241,13 +242,14 @@ int cq_case_indicators(const float* t, const float* c, const float* row_scale, c
  *   "no_pdl"      1: no programmatic dependent launch (quantize pass and diagnostics passes)
  *   "no_stage"    1: the quantize pass loads rows straight into registers instead of staging them in shared memory
  *                    with bulk copies; the weight quantizer uses plain loads for long rows too
- *   "no_small"    1: small matrices (up to 8 column strips of 2048 columns and 32 rows per cluster CTA) take the
- *                    three launches too instead of the single thread-block-cluster launch
+ *   "no_small"    1: decode-sized matrices (up to 8192 columns and 16-32 rows) take the three launches too
+ *                    instead of the single thread-block-cluster launch
  * value <= 0 restores the built-in choice.  Returns CQ_OK or CQ_ERR_SHAPE (unknown key). */
 int cq_set_tuning(const char* key, int value);
 
-/* Health check.  The quantize pass, the diagnostics passes (cq_remove_kernel, cq_kernel_count_x) and the
- * weight quantizer on long rows wait for their asynchronous row copies with a bounded number of polls;
+/* Health check.  The quantize pass, the single-launch path for small matrices, the diagnostics passes
+ * (cq_remove_kernel, cq_kernel_count_x) and the weight quantizer on long rows wait for their asynchronous
+ * row copies with a bounded number of polls;
  * if a wait ever gives up, a device flag is raised (results of that call are then undefined).  This
  * copies the flag of the current device to *fault_host (0 = never happened).  Synchronises the device. */
 int cq_stage_fault(unsigned int* fault_host);
