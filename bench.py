@@ -42,8 +42,8 @@ HOOK_EVERY = 8
 
 # DRAM traffic of the quantize pass from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum
 # per launch), valid only for the kernel sources whose digest is recorded with it.
-NCU_TRAFFIC = {"sources_sha256": "1b50d8e99192c8f7aeb941b244c4254a84417d939707a655caef3473b96b9448",
-               "bytes_per_launch": 527887360}   # 235,210,240 read + 292,677,120 written
+NCU_TRAFFIC = {"sources_sha256": "60e94867662c10a56b051acdb34ed74b9e930e14c7bf2328cb23d22729711be1",
+               "bytes_per_launch": 530871296}   # 235,185,920 read + 295,685,376 written
 
 
 def kernel_sources_digest() -> str:
