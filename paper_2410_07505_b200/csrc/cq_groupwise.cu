@@ -8,11 +8,17 @@
 
 namespace cq {
 
-constexpr int kVecPerThread = 4;
+#ifndef CQ_K7_VEC
+#define CQ_K7_VEC 4
+#endif
+#ifndef CQ_K7_MIN_CTAS
+#define CQ_K7_MIN_CTAS 1
+#endif
+constexpr int kVecPerThread = CQ_K7_VEC;
 
 // LANES = g / 8 (a power of two <= 32).  Groups never straddle a stored row (C % g == 0).
 template <int DT, int BITS, int DEQ, bool CODES, int LANES>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, CQ_K7_MIN_CTAS)
 k7_weight_groups(const uint4* __restrict__ W, int64_t nvec, int C8, int64_t ld8,
                  void* __restrict__ codes, float* __restrict__ scale, void* __restrict__ deq,
                  unsigned long long* __restrict__ zero_count) {
