@@ -141,6 +141,11 @@ def whole_job_gbs(elements_per_rank: int, steps: int, world: int, max_ms: float)
     return BYTES_PER_ELEMENT_STEP * elements_per_rank * steps * world / (max_ms * 1e-3) / 1e9
 
 
+def workload_name(cfg) -> str:
+    return (f"{cfg.name} {cfg.T}x{cfg.I} bf16 (LLaMA-70B MLP input), INT{BITS} codes + bf16 dequant + zero count, "
+            f"alpha={ALPHA}")
+
+
 def run_reference(args) -> None:
     """The oracle, as it stands, on the host cores: each step is a bounded sample of the workload."""
     rank = int(os.environ.get("RANK", "0"))
@@ -164,7 +169,7 @@ def run_reference(args) -> None:
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{cfg.name} {rows}x{cfg.I} bf16 sample, INT{BITS}, alpha={ALPHA}"},
+        "config": {"workload": workload_name(cfg), "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -334,7 +339,7 @@ def main() -> None:
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
         "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{cfg.name} {T}x{I} bf16 (LLaMA-70B MLP input), INT{BITS} codes + bf16 dequant + zero count, alpha={ALPHA}",
+        "config": {"workload": workload_name(cfg),
                    "l2": "flushed between steps (256 MiB write, untimed); X (235 MB) also exceeds the 126 MB L2",
                    "timing": "CUDA events per step on the launch stream, summed; max over ranks",
                    "bytes_per_element": BYTES_PER_ELEMENT_STEP, "per_rank": "independent matrices, no collective"},
