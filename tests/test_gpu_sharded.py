@@ -133,3 +133,23 @@ def test_column_blocks_equal_the_whole_matrix(mods, shape, cuts, dtype, bits, al
         codes = parity.unpack_int4(codes, T, j1 - j0) if bits == 4 else codes.view(np.int8)
         assert np.array_equal(codes, ref.codes[:, j0:j1])
         assert np.array_equal(bits_of(o.deq).reshape(T, j1 - j0), ref.deq16[:, j0:j1])
+
+
+def test_block_entry_points_report_bad_arguments(mods):
+    cq, _ = mods
+    L = cq.lib()
+    X = to_dev(wl.small_matrix(8, 64, "bf16", 1), "bf16")
+    ws = torch.empty(cq.workspace_bytes(8, 64), dtype=torch.uint8, device="cuda")
+    v = torch.ones(64, dtype=torch.float32, device="cuda")
+    assert L.cq_vector_max(None, None, 0, None) == 0                     # nothing to do
+    assert L.cq_vector_max(None, cq._ptr(v), 64, None) == 1              # CQ_ERR_NULL
+    assert L.cq_vector_max(cq._ptr(v), cq._ptr(v), -1, None) == 2        # CQ_ERR_SHAPE
+    rc = L.cq_quantize_act_given(cq._ptr(X), 1, 8, 64, 64, 0.15, 8, None, cq._ptr(v), None, None, None, None, 1, None,
+                                 cq._ptr(ws), ws.numel(), None)
+    assert rc == 1                                                       # t missing
+    rc = L.cq_quantize_act_given(cq._ptr(X), 1, 8, 64, 64, 1.5, 8, cq._ptr(v), cq._ptr(v), None, None, None, None, 1, None,
+                                 cq._ptr(ws), ws.numel(), None)
+    assert rc == 5                                                       # alpha out of range
+    with pytest.raises(ValueError):
+        cq.vector_max_(v, v[:32])
+    torch.cuda.synchronize()
