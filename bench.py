@@ -370,8 +370,17 @@ def main() -> None:
         orc.quantize_act(X, cfg.dtype, ALPHA, BITS, want_deq32=False)
         reps += 1
     dt = time.perf_counter() - t0
+    all_threads = orc.num_threads()
+    Xs = np.ascontiguousarray(X[:256])                                   # one core: a 256-row sample is enough
+    orc.set_num_threads(1)
+    t1 = time.perf_counter()
+    orc.quantize_act(Xs, cfg.dtype, ALPHA, BITS, want_deq32=False)
+    dt1 = time.perf_counter() - t1
+    orc.set_num_threads(all_threads)
     out["cpu_baseline"] = {"value": BYTES_PER_ELEMENT_STEP * X.size * reps / dt / 1e9, "unit": UNIT,
-                           "cores": orc.num_threads(), "kind": "oracle",
+                           "cores": all_threads, "kind": "oracle",
+                           "single_thread_value": BYTES_PER_ELEMENT_STEP * Xs.size / dt1 / 1e9,
+                           "host_cores": os.cpu_count(),
                            "sample": f"the whole workload matrix ({T}x{I}), {reps} oracle quantize_act calls "
                                      f"(t, c, codes, bf16 dequant, count) in {dt:.2f} s wall on {orc.num_threads()} threads"}
     print(json.dumps(out))

@@ -414,6 +414,15 @@ void cqo_case_indicators(const float* t, const float* c, const float* a, const f
     out[1] = n_smaller;
 }
 
+/* Number of OpenMP threads later calls may use (timing only: results do not depend on it).  n < 1 is ignored. */
+void cqo_set_num_threads(int n) {
+#ifdef _OPENMP
+    if (n >= 1) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
 int cqo_num_threads(void) {
     int n = 1;
 #ifdef _OPENMP

@@ -49,6 +49,11 @@ def num_threads() -> int:
     return int(lib().cqo_num_threads())
 
 
+def set_num_threads(n: int) -> None:
+    """OpenMP threads for later calls (for timing the oracle on one core and on all; results are unaffected)."""
+    lib().cqo_set_num_threads(C.c_int(int(n)))
+
+
 def decode16(bits: np.ndarray, dtype: str) -> np.ndarray:
     bits = np.ascontiguousarray(bits, dtype=np.uint16)
     out = np.empty(bits.shape, dtype=np.float32)
