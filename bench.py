@@ -42,8 +42,8 @@ HOOK_EVERY = 8
 
 # DRAM traffic of the quantize pass from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum
 # per launch), valid only for the kernel sources whose digest is recorded with it.
-NCU_TRAFFIC = {"sources_sha256": "60e94867662c10a56b051acdb34ed74b9e930e14c7bf2328cb23d22729711be1",
-               "bytes_per_launch": 530871296}   # 235,185,920 read + 295,685,376 written
+NCU_TRAFFIC = {"sources_sha256": "626eb9ce7da18000539bdd22ddae4b17cb91e80b70835ad46d56c63bbe803dca",
+               "bytes_per_launch": 527777280}   # 235,185,920 read + 292,591,360 written
 
 
 def kernel_sources_digest() -> str:

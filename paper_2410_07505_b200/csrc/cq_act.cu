@@ -637,9 +637,10 @@ static bool launch_k3_staged(const Plan& p, const K3Args& k, cudaStream_t st) {
 template <int DT, int BITS, int DEQ, bool CODES, bool COUNT>
 static void launch_k3_one(const Plan& p, const K3Args& k, cudaStream_t st) {
     if (!g_tune_no_stage) {
-        // matrices that stream from HBM run two CTAs per SM, those L2 can hold run three
+        // matrices that stream from HBM run two CTAs per SM, those L2 can hold run three (INT8; with INT4
+        // codes the two-CTA build is the faster one at every size measured)
         const int64_t bytes = k.T * k.ld8 * 16;
-        int mode = bytes > (int64_t(120) << 20) ? 2 : 3;
+        int mode = (bytes > (int64_t(120) << 20) || BITS == 4) ? 2 : 3;
         if (g_tune_k3_ctas == 2 || g_tune_k3_ctas == 3) mode = g_tune_k3_ctas;
         const bool ok = mode == 2 ? launch_k3_staged<DT, BITS, DEQ, CODES, COUNT, 2>(p, k, st)
                                   : launch_k3_staged<DT, BITS, DEQ, CODES, COUNT, 3>(p, k, st);
