@@ -88,6 +88,9 @@ size_t cq_workspace_bytes(int64_t T, int64_t I);
  *   zero_count out  device uint64, number of zero codes = |K(CQ)|; nullable
  *   workspace  in   device, 256-byte aligned, >= cq_workspace_bytes(T, I); contents undefined after
  * T == 0 or I == 0 is valid: only zero_count (= 0) is written.
+ * The call only enqueues kernels (and at most two small device-to-device copies) on `stream`; after one
+ * ordinary call per shape on a device (which settles the kernels' launch attributes) it can be captured
+ * in a CUDA graph and replayed.
  */
 int cq_quantize_act(const void* X, int dtype, int64_t T, int64_t I, int64_t ld,
                     double alpha, int bits,

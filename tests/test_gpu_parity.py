@@ -190,6 +190,33 @@ def test_small_matrices_one_launch_and_three_launches(cq, shape, dtype):
     assert cq.stage_fault() == 0
 
 
+@pytest.mark.parametrize("shape", [(300, 2056), (16, 4096), (513, 776)])
+def test_public_call_replays_from_a_cuda_graph(cq, shape):
+    """After one ordinary call (which settles the per-kernel launch attributes) the call only enqueues kernels,
+    so it can be captured once and replayed on new contents of the same buffers."""
+    T, I = shape
+    X1 = wl.small_matrix(T, I, "bf16", 31, outlier_cols=3, zero_frac=0.02)
+    X2 = wl.small_matrix(T, I, "bf16", 32, outlier_cols=3, zero_frac=0.02)
+    Xd = to_dev(X1, "bf16")
+    buf = cq.ActBuffers(T, I, Xd.dtype, 8)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        cq.quantize_act(Xd, 0.15, 8, buffers=buf)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        cq.quantize_act(Xd, 0.15, 8, buffers=buf)
+    for X in (X1, X2, X1):
+        Xd.copy_(to_dev(X, "bf16"))
+        for b in (buf.codes, buf.deq, buf.t, buf.c, buf.row_scale, buf.col_scale):
+            b.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        parity.check_act(X, "bf16", 0.15, 8, t=buf.t.cpu().numpy(), c=buf.c.cpu().numpy(), a=buf.row_scale.cpu().numpy(),
+                         b=buf.col_scale.cpu().numpy(), codes=buf.codes.cpu().numpy(), deq=bits_of(buf.deq),
+                         zero_count=int(buf.zero_count.item()))
+
+
 def test_launch_without_programmatic_dependent_launch_gives_the_same_results(cq):
     try:
         cq.set_tuning("no_pdl", 1)
