@@ -86,17 +86,53 @@ def time_extra_ops(Xd: torch.Tensor, alpha: float, flush, iters: int) -> dict:
             "share_c_ge_t": ind[0] / n, "share_bound_smaller": ind[1] / n}
 
 
+def time_decode_shapes(flush, iters: int) -> None:
+    """Decode-sized matrices: CUDA-event time of one call after an L2 flush, wall time per call of 200 calls issued
+    back to back (host included), for the single-launch path and the three launches, and per replay of a graph."""
+    import time
+    for T, I in ((1, 4096), (16, 4096), (16, 8192), (32, 2048), (64, 8192)):
+        Xd = _dev(wl.small_matrix(T, I, "bf16", 3, outlier_cols=4), "bf16")
+        buf = cq.ActBuffers(T, I, Xd.dtype, 8)
+        row = {"shape": [T, I], "dtype": "bf16", "bits": 8}
+        for key, no_small in (("one_launch", 0), ("three_launches", 1)):
+            cq.set_tuning("no_small", no_small)
+            cold = _time(lambda: cq.quantize_act(Xd, 0.15, 8, buffers=buf), flush, iters)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for _ in range(200):
+                cq.quantize_act(Xd, 0.15, 8, buffers=buf)
+            torch.cuda.synchronize()
+            row[key] = {"us_l2_flushed": round(cold, 1), "us_per_call_back_to_back": round((time.perf_counter() - t0) / 200 * 1e6, 1)}
+        cq.set_tuning("no_small", 0)
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            cq.quantize_act(Xd, 0.15, 8, buffers=buf)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(200):
+            graph.replay()
+        torch.cuda.synchronize()
+        row["graph_replay_us"] = round((time.perf_counter() - t0) / 200 * 1e6, 1)
+        print(json.dumps(row), flush=True)
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--iters", type=int, default=30)
     ap.add_argument("--layers", type=int, default=0, help="layers of the 80-layer sweep to run (0 = skip)")
     ap.add_argument("--alpha", type=float, default=0.15)
+    ap.add_argument("--decode", action="store_true", help="time decode-sized matrices through the single-launch path, "
+                    "the three launches and a CUDA-graph replay, then exit")
     ap.add_argument("--only", default="", help="comma-separated config names (e.g. llama70b_mlp,weight_8192x28672): "
                     "time only these (keeps a profiler capture short)")
     args = ap.parse_args()
     only = set(filter(None, args.only.split(",")))
     cq.lib()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    if args.decode:
+        time_decode_shapes(flush, args.iters)
+        return
 
     for name, cfg in wl.ACT_CONFIGS.items():
         if only and name not in only:
