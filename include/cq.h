@@ -87,7 +87,9 @@ size_t cq_workspace_bytes(int64_t T, int64_t I);
  *   deq        out  device [T*I] of deq_dtype (X's dtype or CQ_F32); nullable
  *   zero_count out  device uint64, number of zero codes = |K(CQ)|; nullable
  *   workspace  in   device, 256-byte aligned, >= cq_workspace_bytes(T, I); contents undefined after
- * T == 0 or I == 0 is valid: only zero_count (= 0) is written.
+ * T == 0 or I == 0 is valid: zero_count = 0, and the vectors of the non-empty dimension are still written
+ * (maxima over nothing are 0: t = 0 or c = 0, with the scale factors that follow from them), so that an empty
+ * row block contributes zeros when the blocks' column maxima are combined.
  * The call only enqueues kernels (and at most two small device-to-device copies) on `stream`; after one
  * ordinary call per shape on a device (which settles the kernels' launch attributes) it can be captured
  * in a CUDA graph and replayed.

@@ -142,16 +142,33 @@ def _workspace(T, I, device):
 
 
 # ----------------------------------------------------------------------------- absmax
-def absmax_rows(X: torch.Tensor) -> torch.Tensor:
+def _f32_vector(out, n: int, device, what: str) -> torch.Tensor:
+    if out is None:
+        return torch.empty(n, dtype=torch.float32, device=device)
+    if out.dtype != torch.float32 or out.numel() != n or not out.is_contiguous() or out.device != device:
+        raise ValueError(f"{what} must be a contiguous float32 vector of {n} elements on {device}")
+    return out
+
+
+def _counts(out, n: int, device, what: str) -> torch.Tensor:
+    """An int64 device tensor of n elements (a scalar for n == 1) that receives 64-bit counts."""
+    if out is None:
+        return torch.zeros((), dtype=torch.int64, device=device) if n == 1 else torch.zeros(n, dtype=torch.int64, device=device)
+    if out.dtype != torch.int64 or out.numel() != n or not out.is_contiguous() or out.device != device:
+        raise ValueError(f"{what} must be a contiguous int64 tensor of {n} element(s) on {device}")
+    return out
+
+
+def absmax_rows(X: torch.Tensor, *, out: torch.Tensor | None = None) -> torch.Tensor:
     T, I, ld = _matrix_args(X)
-    t = torch.empty(T, dtype=torch.float32, device=X.device)
+    t = _f32_vector(out, T, X.device, "out")
     _check(lib().cq_absmax_rows(_ptr(X), _DT[X.dtype], T, I, ld, _ptr(t), _stream()), "cq_absmax_rows")
     return t
 
 
-def absmax_cols(X: torch.Tensor) -> torch.Tensor:
+def absmax_cols(X: torch.Tensor, *, out: torch.Tensor | None = None) -> torch.Tensor:
     T, I, ld = _matrix_args(X)
-    c = torch.empty(I, dtype=torch.float32, device=X.device)
+    c = _f32_vector(out, I, X.device, "out")
     _check(lib().cq_absmax_cols(_ptr(X), _DT[X.dtype], T, I, ld, _ptr(c), _stream()), "cq_absmax_cols")
     return c
 
@@ -161,8 +178,8 @@ def absmax_rows_cols(X: torch.Tensor, *, workspace: torch.Tensor | None = None, 
     cq_quantize_act is used (partial maxima in the workspace, no atomics: faster on large matrices);
     without one, cq_absmax_rows_cols.  `out` = (t, c) tensors to fill."""
     T, I, ld = _matrix_args(X)
-    t, c = out if out is not None else (torch.empty(T, dtype=torch.float32, device=X.device),
-                                        torch.empty(I, dtype=torch.float32, device=X.device))
+    t = _f32_vector(out[0] if out is not None else None, T, X.device, "out[0]")
+    c = _f32_vector(out[1] if out is not None else None, I, X.device, "out[1]")
     if workspace is None:
         _check(lib().cq_absmax_rows_cols(_ptr(X), _DT[X.dtype], T, I, ld, _ptr(t), _ptr(c), _stream()),
                "cq_absmax_rows_cols")
@@ -210,6 +227,24 @@ class ActBuffers:
         self.workspace = _workspace(T, I, dev)
 
 
+def _check_act_buffers(b: "ActBuffers", T: int, I: int, dtype: torch.dtype, bits: int, where: str) -> None:
+    """The kernels trust the sizes they are told: refuse buffers made for another shape, dtype or bit width."""
+    def bad(what):
+        raise ValueError(f"{where}: buffers.{what} does not match a {T} x {I} {dtype} matrix quantized to {bits} bits")
+    for name, n in (("t", T), ("c", I), ("row_scale", T), ("col_scale", I)):
+        v = getattr(b, name)
+        if v is not None and (v.dtype != torch.float32 or v.numel() != n or not v.is_contiguous()):
+            bad(name)
+    if b.codes is not None:
+        want = T * I if bits == 8 else T * (I // 2)
+        if b.codes.element_size() != 1 or b.codes.numel() != want or not b.codes.is_contiguous():
+            bad("codes")
+    if b.deq is not None and (b.deq.dtype not in (dtype, torch.float32) or b.deq.numel() != T * I or not b.deq.is_contiguous()):
+        bad("deq")
+    if b.zero_count is not None and (b.zero_count.dtype != torch.int64 or b.zero_count.numel() != 1):
+        bad("zero_count")
+
+
 def quantize_act(X: torch.Tensor, alpha: float = 0.15, bits: int = 8, *, codes: bool = True,
                  deq: bool = True, deq_dtype: torch.dtype | None = None, count: bool = True,
                  buffers: ActBuffers | None = None) -> ActQuant:
@@ -219,6 +254,7 @@ def quantize_act(X: torch.Tensor, alpha: float = 0.15, bits: int = 8, *, codes: 
         raise CQError(6, "cq_quantize_act")
     b = buffers or ActBuffers(T, I, X.dtype, bits, codes=codes, deq=deq, deq_dtype=deq_dtype, count=count,
                               device=X.device)
+    _check_act_buffers(b, T, I, X.dtype, bits, "quantize_act")
     deq_dt = _DT[b.deq.dtype] if b.deq is not None else _DT[X.dtype]
     st = lib().cq_quantize_act(_ptr(X), _DT[X.dtype], T, I, ld, float(alpha), int(bits), _ptr(b.t), _ptr(b.c),
                                _ptr(b.row_scale), _ptr(b.col_scale), _ptr(b.codes), _ptr(b.deq), deq_dt,
@@ -250,6 +286,7 @@ def quantize_act_given(X: torch.Tensor, t: torch.Tensor, c: torch.Tensor, alpha:
         raise ValueError("t must be float32[T] and c float32[I]")
     b = buffers or ActBuffers(T, I, X.dtype, bits, codes=codes, deq=deq, deq_dtype=deq_dtype, count=count,
                               device=X.device)
+    _check_act_buffers(b, T, I, X.dtype, bits, "quantize_act_given")
     deq_dt = _DT[b.deq.dtype] if b.deq is not None else _DT[X.dtype]
     st = lib().cq_quantize_act_given(_ptr(X), _DT[X.dtype], T, I, ld, float(alpha), int(bits), _ptr(t), _ptr(c),
                                      _ptr(b.row_scale), _ptr(b.col_scale), _ptr(b.codes), _ptr(b.deq), deq_dt,
@@ -267,6 +304,7 @@ def quantize_act_noalloc(X: torch.Tensor, alpha: float = 0.15, bits: int = 8, *,
     the array up and should come before any stream capture."""
     T, I, ld = _matrix_args(X)
     b = buffers
+    _check_act_buffers(b, T, I, X.dtype, bits, "quantize_act_noalloc")
     deq_dt = _DT[b.deq.dtype] if b.deq is not None else _DT[X.dtype]
     st = lib().cq_quantize_act_noalloc(_ptr(X), _DT[X.dtype], T, I, ld, float(alpha), int(bits), _ptr(b.t), _ptr(b.c),
                                        _ptr(b.row_scale), _ptr(b.col_scale), _ptr(b.codes), _ptr(b.deq), deq_dt,
@@ -322,24 +360,33 @@ def quantize_act_host(X_host: torch.Tensor, alpha: float = 0.15, bits: int = 8, 
 
 
 def dequantize(codes: torch.Tensor, bits: int, T: int, I: int, row_scale: torch.Tensor, col_scale: torch.Tensor,
-               out_dtype: torch.dtype = torch.float32) -> torch.Tensor:
-    out = torch.empty((T, I), dtype=out_dtype, device=codes.device)
+               out_dtype: torch.dtype = torch.float32, *, out: torch.Tensor | None = None) -> torch.Tensor:
+    if out is None:
+        out = torch.empty((T, I), dtype=out_dtype, device=codes.device)
+    elif out.dtype != out_dtype or out.numel() != T * I or not out.is_contiguous():
+        raise ValueError("out must be a contiguous [T, I] tensor of out_dtype")
+    if row_scale.numel() != T or col_scale.numel() != I or codes.numel() * codes.element_size() != (T * I if bits == 8 else T * (I // 2)):
+        raise ValueError("codes / scale vectors do not match T, I and bits")
     _check(lib().cq_dequantize(_ptr(codes), int(bits), T, I, _ptr(row_scale), _ptr(col_scale), _ptr(out),
                                _DT[out_dtype], _stream()), "cq_dequantize")
     return out
 
 
-def kernel_count(codes: torch.Tensor, bits: int, T: int, I: int) -> torch.Tensor:
-    count = torch.zeros((), dtype=torch.int64, device=codes.device)
+def kernel_count(codes: torch.Tensor, bits: int, T: int, I: int, *, count: torch.Tensor | None = None) -> torch.Tensor:
+    count = _counts(count, 1, codes.device, "count")
+    if codes.numel() * codes.element_size() != (T * I if bits == 8 else T * (I // 2)):
+        raise ValueError("codes do not match T, I and bits")
     _check(lib().cq_kernel_count(_ptr(codes), int(bits), T, I, _ptr(count), _stream()), "cq_kernel_count")
     return count
 
 
 def kernel_count_x(X: torch.Tensor, alpha: float, bits: int, t: torch.Tensor, c: torch.Tensor,
-                   workspace: torch.Tensor | None = None) -> torch.Tensor:
+                   workspace: torch.Tensor | None = None, *, count: torch.Tensor | None = None) -> torch.Tensor:
     T, I, ld = _matrix_args(X)
+    if t.dtype != torch.float32 or c.dtype != torch.float32 or t.numel() != T or c.numel() != I:
+        raise ValueError("t must be float32[T] and c float32[I]")
     ws = workspace if workspace is not None else _workspace(T, I, X.device)
-    count = torch.zeros((), dtype=torch.int64, device=X.device)
+    count = _counts(count, 1, X.device, "count")
     _check(lib().cq_kernel_count_x(_ptr(X), _DT[X.dtype], T, I, ld, float(alpha), int(bits), _ptr(t), _ptr(c),
                                    _ptr(count), _ptr(ws), ws.numel(), _stream()), "cq_kernel_count_x")
     return count
@@ -352,6 +399,21 @@ class WeightQuant:
     deq: torch.Tensor | None
     zero_count: torch.Tensor | None
     bits: int
+
+
+def _check_weight_out(out: "WeightQuant", R: int, Cc: int, n_scales: int, dtype: torch.dtype, bits: int, where: str) -> None:
+    def bad(what):
+        raise ValueError(f"{where}: out.{what} does not match a {R} x {Cc} {dtype} matrix quantized to {bits} bits")
+    if out.scale is not None and (out.scale.dtype != torch.float32 or out.scale.numel() != n_scales or not out.scale.is_contiguous()):
+        bad("scale")
+    if out.codes is not None:
+        want = R * Cc if bits == 8 else R * (Cc // 2)
+        if out.codes.element_size() != 1 or out.codes.numel() != want or not out.codes.is_contiguous():
+            bad("codes")
+    if out.deq is not None and (out.deq.dtype not in (dtype, torch.float32) or out.deq.numel() != R * Cc or not out.deq.is_contiguous()):
+        bad("deq")
+    if out.zero_count is not None and (out.zero_count.dtype != torch.int64 or out.zero_count.numel() != 1):
+        bad("zero_count")
 
 
 def quantize_weight_per_channel(W: torch.Tensor, bits: int = 8, *, codes: bool = True, deq: bool = True,
@@ -370,6 +432,7 @@ def quantize_weight_per_channel(W: torch.Tensor, bits: int = 8, *, codes: bool =
         out = WeightQuant(torch.empty(R, dtype=torch.float32, device=dev), codes_t,
                           torch.empty((R, Cc), dtype=deq_dtype or W.dtype, device=dev) if deq else None,
                           torch.zeros((), dtype=torch.int64, device=dev) if count else None, bits)
+    _check_weight_out(out, R, Cc, R, W.dtype, bits, "quantize_weight_per_channel")
     deq_dt = _DT[out.deq.dtype] if out.deq is not None else _DT[W.dtype]
     st = lib().cq_quantize_weight_per_channel(_ptr(W), _DT[W.dtype], R, Cc, ld, int(bits), _ptr(out.codes),
                                               _ptr(out.scale), _ptr(out.deq), deq_dt, _ptr(out.zero_count),
@@ -394,6 +457,8 @@ def quantize_weight_groupwise(W: torch.Tensor, group: int = 128, bits: int = 4, 
         out = WeightQuant(torch.empty(n_groups, dtype=torch.float32, device=dev), codes_t,
                           torch.empty((R, Cc), dtype=deq_dtype or W.dtype, device=dev) if deq else None,
                           torch.zeros((), dtype=torch.int64, device=dev) if count else None, bits)
+    if group > 0 and Cc % group == 0:
+        _check_weight_out(out, R, Cc, R * (Cc // group), W.dtype, bits, "quantize_weight_groupwise")
     deq_dt = _DT[out.deq.dtype] if out.deq is not None else _DT[W.dtype]
     st = lib().cq_quantize_weight_groupwise(_ptr(W), _DT[W.dtype], R, Cc, ld, int(group), int(bits), _ptr(out.codes),
                                             _ptr(out.scale), _ptr(out.deq), deq_dt, _ptr(out.zero_count), _stream())
@@ -401,23 +466,27 @@ def quantize_weight_groupwise(W: torch.Tensor, group: int = 128, bits: int = 4, 
     return out
 
 
-def case_indicators(r: ActQuant) -> torch.Tensor:
+def case_indicators(r: ActQuant, *, counts: torch.Tensor | None = None) -> torch.Tensor:
     """Table 1 indicators of a quantize_act result: int64[2] on the device,
     (#pairs with c_j >= t_i, #pairs whose CrossQuant zero bound is below the per-token bound)."""
-    counts = torch.zeros(2, dtype=torch.int64, device=r.t.device)
+    counts = _counts(counts, 2, r.t.device, "counts")
     _check(lib().cq_case_indicators(_ptr(r.t), _ptr(r.c), _ptr(r.row_scale), _ptr(r.col_scale), r.t.numel(),
                                     r.c.numel(), int(r.bits), _ptr(counts), _stream()), "cq_case_indicators")
     return counts
 
 
 def remove_kernel(X: torch.Tensor, alpha: float = 0.15, bits: int = 8, bound_scale: float = 1.0,
-                  workspace: torch.Tensor | None = None):
+                  workspace: torch.Tensor | None = None, *, out: torch.Tensor | None = None,
+                  counts: torch.Tensor | None = None):
     """Remove-Kernel operator: returns (X with the kernel elements set to +0 and the rest untouched,
     int64[3] device counts: removed, per-token kernel size, CrossQuant kernel size)."""
     T, I, ld = _matrix_args(X)
     ws = workspace if workspace is not None else _workspace(T, I, X.device)
-    out = torch.empty((T, I), dtype=X.dtype, device=X.device)
-    counts = torch.zeros(3, dtype=torch.int64, device=X.device)
+    if out is None:
+        out = torch.empty((T, I), dtype=X.dtype, device=X.device)
+    elif out.dtype != X.dtype or tuple(out.shape) != (T, I) or not out.is_contiguous():
+        raise ValueError("out must be a contiguous [T, I] tensor of X's dtype")
+    counts = _counts(counts, 3, X.device, "counts")
     _check(lib().cq_remove_kernel(_ptr(X), _DT[X.dtype], T, I, ld, float(alpha), int(bits), float(bound_scale), _ptr(out),
                                   _ptr(counts), _ptr(ws), ws.numel(), _stream()), "cq_remove_kernel")
     return out, counts

@@ -247,6 +247,20 @@ k2_scales_from_vectors(int64_t T, int64_t I, const float* __restrict__ t_in, con
     }
 }
 
+// An empty matrix (no rows or no columns) still has scale vectors in its non-empty dimension: those of the
+// supplied maxima, or of 0 (the maximum over nothing) where none are supplied.  Every pointer may be null.
+__global__ void __launch_bounds__(kThreads)
+k2_scales_of_empty(int64_t T, int64_t I, const float* __restrict__ t_in, const float* __restrict__ c_in,
+                   double alpha, int qmax, float* __restrict__ a, float* __restrict__ b) {
+    const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    float f, r;
+    if (idx < T) {
+        if (a != nullptr) { row_scale_of(t_in != nullptr ? t_in[idx] : 0.0f, alpha, qmax, f, r); a[idx] = f; }
+    } else if (idx - T < I) {
+        if (b != nullptr) { col_scale_of(c_in != nullptr ? c_in[idx - T] : 0.0f, alpha, qmax, f, r); b[idx - T] = f; }
+    }
+}
+
 // acc_j = max(acc_j, v_j): combines the maxima of row blocks of one matrix (magnitudes, so never NaN-ordered
 // surprises: fmaxf of two non-negative floats).
 __global__ void __launch_bounds__(kThreads)
@@ -706,8 +720,19 @@ int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
                            t_given, c_given})
         if (f != nullptr && !aligned(f, 4)) return CQ_ERR_ALIGN;
     if (T == 0 || I == 0) {
+        // Nothing to quantize, but the vectors of the non-empty dimension are still results: maxima over nothing
+        // are 0 (a row block without rows must contribute zeros to the combined column maxima).
         if (zero_count != nullptr && cudaMemsetAsync(zero_count, 0, sizeof(unsigned long long), st) != cudaSuccess)
             return CQ_ERR_CUDA;
+        if (t != nullptr && T > 0 && cudaMemsetAsync(t, 0, sizeof(float) * T, st) != cudaSuccess) return CQ_ERR_CUDA;
+        if (c != nullptr && I > 0 && cudaMemsetAsync(c, 0, sizeof(float) * I, st) != cudaSuccess) return CQ_ERR_CUDA;
+        float* a_out = T > 0 ? row_scale : nullptr;
+        float* b_out = I > 0 ? col_scale : nullptr;
+        if (a_out != nullptr || b_out != nullptr) {
+            const unsigned blocks = static_cast<unsigned>((T + I + kThreads - 1) / kThreads);
+            k2_scales_of_empty<<<blocks, kThreads, 0, st>>>(T, I, t_given, c_given, alpha, (1 << (bits - 1)) - 1, a_out, b_out);
+            return launch_status();
+        }
         return CQ_OK;
     }
     Plan p = make_plan(T, I);

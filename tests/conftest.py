@@ -18,3 +18,17 @@ def _oracle_built():
     from oracle import build as oracle_build
     oracle_build.build()
     yield
+
+
+@pytest.fixture(scope="module")
+def cq():
+    """The binding module behind guard bands: every output a GPU test receives sits between canary bytes that are
+    checked after each call (tests/guards.py).  Fails, rather than skips, without a CUDA device."""
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("the gpu tests need a CUDA device")
+    from paper_2410_07505_b200 import build, cq as _cq
+    build.build()
+    _cq.lib()
+    from guards import Guarded
+    return Guarded(_cq)

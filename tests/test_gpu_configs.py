@@ -10,7 +10,7 @@ from oracle import cq_oracle as orc
 from oracle import parity
 from paper_2410_07505_b200 import workloads as wl
 
-from test_gpu_parity import bits_of, cq, to_dev  # noqa: F401  (cq is a fixture)
+from test_gpu_parity import bits_of, to_dev
 
 pytestmark = pytest.mark.gpu
 

@@ -14,16 +14,6 @@ pytestmark = pytest.mark.gpu
 TORCH_DT = {"f16": torch.float16, "bf16": torch.bfloat16}
 
 
-@pytest.fixture(scope="module")
-def cq():
-    if not torch.cuda.is_available():
-        pytest.fail("the gpu tests need a CUDA device")
-    from paper_2410_07505_b200 import build, cq as _cq
-    build.build()
-    _cq.lib()
-    return _cq
-
-
 def to_dev(bits: np.ndarray, dtype: str) -> torch.Tensor:
     return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(TORCH_DT[dtype]).cuda()
 

@@ -15,13 +15,13 @@ TORCH_DT = {"f16": torch.float16, "bf16": torch.bfloat16}
 
 
 @pytest.fixture(scope="module")
-def mods():
-    if not torch.cuda.is_available():
-        pytest.fail("the gpu tests need a CUDA device")
-    from paper_2410_07505_b200 import build, cq, sharded
-    build.build()
-    cq.lib()
-    return cq, sharded
+def mods(cq):
+    """(binding behind guard bands, the sharded module made to allocate and call through the same guarded binding)."""
+    from paper_2410_07505_b200 import sharded
+    plain = sharded.cq
+    sharded.cq = cq
+    yield cq, sharded
+    sharded.cq = plain
 
 
 def to_dev(bits: np.ndarray, dtype: str) -> torch.Tensor:
@@ -153,3 +153,29 @@ def test_block_entry_points_report_bad_arguments(mods):
     with pytest.raises(ValueError):
         cq.vector_max_(v, v[:32])
     torch.cuda.synchronize()
+
+
+def test_an_empty_row_block_contributes_zeros_to_the_combined_maxima(mods):
+    """A rank or chunk without rows (T < world size) still hands a column-maximum vector to the exchange: it must be
+    zeros, whatever the buffer held before, and the other blocks' results must equal the whole matrix's."""
+    cq, sharded = mods
+    X = wl.small_matrix(5, 264, "bf16", 17, outlier_cols=2)
+    Xd = to_dev(X, "bf16")
+    b = cq.ActBuffers(0, 264, Xd.dtype, 8)
+    b.c.fill_(float("nan"))
+    b.col_scale.fill_(float("nan"))
+    _, c = cq.absmax_rows_cols(Xd[0:0], workspace=b.workspace, out=(b.t, b.c))
+    torch.cuda.synchronize()
+    assert not c.any() and c.numel() == 264
+    r = cq.quantize_act(Xd[0:0], 0.15, 8, buffers=b)                        # scale factors of c = 0: zeros too
+    assert int(r.zero_count.item()) == 0 and not r.col_scale.any()
+    for alpha in (0.15, 1.0):
+        outs, total = sharded.quantize_act_chunked([Xd[:3], Xd[3:3], Xd[3:]], alpha, 8)
+        torch.cuda.synchronize()
+        assert torch.equal(outs[1].c, outs[0].c)
+        check_blocks(X, "bf16", alpha, 8, [outs[0], outs[2]], total)
+    # the same for a column block without columns: its row maxima are zeros
+    b = cq.ActBuffers(5, 0, Xd.dtype, 8)
+    b.t.fill_(float("nan"))
+    t, _ = cq.absmax_rows_cols(Xd[:, 0:0], workspace=b.workspace, out=(b.t, b.c))
+    assert not t.any() and t.numel() == 5

@@ -6,7 +6,9 @@ pool, or the host application bans allocation on its hot path), so this entry po
 in a fixed array inside the library.  Every call reuses that array and finds the previous call's
 contents in it; the test therefore runs each case twice in a row, and on different shapes back to back,
 and compares every output bit for bit with the ordinary entry point (the tolerance the other parity
-tests use for identical arithmetic).  The file name makes pytest collect it last.
+tests use for identical arithmetic); one case is also checked against the CPU oracle directly, and the
+amount of free device memory must not move across the calls.  The outputs sit between guard bands
+(tests/guards.py).  The file name makes pytest collect it last.
 """
 from __future__ import annotations
 
@@ -14,21 +16,12 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import parity
 from paper_2410_07505_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
 
 TORCH_DT = {"f16": torch.float16, "bf16": torch.bfloat16}
-
-
-@pytest.fixture(scope="module")
-def cq():
-    if not torch.cuda.is_available():
-        pytest.fail("the gpu tests need a CUDA device")
-    from paper_2410_07505_b200 import build, cq as _cq
-    build.build()
-    _cq.lib()
-    return _cq
 
 
 def _dev(bits, dtype):
@@ -57,13 +50,35 @@ def test_noalloc_matches_the_ordinary_entry_point_on_repeated_calls(cq):
             r = cq.quantize_act_noalloc(Xd, alpha, bits, buffers=out)
             torch.cuda.synchronize()
             _same(r, ref)
+        del ref, out
+
+
+def test_noalloc_matches_the_oracle_and_allocates_nothing(cq):
+    T, I, dtype, bits, alpha = 515, 2056, "bf16", 8, 0.15
+    X = wl.small_matrix(T, I, dtype, 4242, outlier_cols=3, zero_frac=0.01)
+    Xd = _dev(X, dtype)
+    out = cq.ActBuffers(T, I, Xd.dtype, bits)
+    L = cq.lib()
+    args = (cq._ptr(Xd), cq._DT[Xd.dtype], T, I, I, alpha, bits, cq._ptr(out.t), cq._ptr(out.c), cq._ptr(out.row_scale),
+            cq._ptr(out.col_scale), cq._ptr(out.codes), cq._ptr(out.deq), cq._DT[Xd.dtype], cq._ptr(out.zero_count), None)
+    assert L.cq_quantize_act_noalloc(*args) == 0           # the first call on this device may look the array up
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for _ in range(3):                                     # straight through the C ABI: no torch allocation in between
+        assert L.cq_quantize_act_noalloc(*args) == 0
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free0, "free device memory changed across a no-allocation call"
+    out.arena.check("cq_quantize_act_noalloc")
+    parity.check_act(X, dtype, alpha, bits, t=out.t.cpu().numpy(), c=out.c.cpu().numpy(), a=out.row_scale.cpu().numpy(),
+                     b=out.col_scale.cpu().numpy(), codes=out.codes.cpu().numpy(),
+                     deq=out.deq.view(torch.int16).cpu().numpy().view(np.uint16), zero_count=int(out.zero_count.item()))
 
 
 def test_noalloc_refuses_shapes_beyond_its_scratch(cq):
     T, I = 3_000_000, 8                                             # three fp32 vectors of 12 MB alone exceed 8 MiB
     assert cq.workspace_bytes(T, I) > cq.NOALLOC_SCRATCH_BYTES
     Xd = torch.zeros((T, I), dtype=torch.bfloat16, device="cuda")
-    out = cq.ActBuffers(8, 8, torch.bfloat16, 8)
+    out = cq.ActBuffers(T, I, torch.bfloat16, 8)
     with pytest.raises(cq.CQError) as e:
         cq.quantize_act_noalloc(Xd, 0.15, 8, buffers=out)
     assert e.value.status == 9
