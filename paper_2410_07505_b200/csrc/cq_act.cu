@@ -13,6 +13,7 @@
 
 #include "cq_common.cuh"
 #include "cq_host.h"
+#include "cq_passes.cuh"
 
 #ifndef CQ_K3_MIN_CTAS
 #define CQ_K3_MIN_CTAS 2
@@ -162,13 +163,7 @@ g1_absmax(const uint16_t* __restrict__ X, int64_t T, int64_t I, int64_t ld, int 
 }
 
 // ============================================================================ scale vectors
-// From the partial maxima of pass 1.  CTAs [0, col_ctas): 64 columns each; thread (vx, grp) reduces every
-// 32nd partial row of vector column vx (8 vector columns x 32 groups per CTA, so even the ~300 partial rows
-// of a narrow matrix cost each thread only ~10 independent loads), shared memory combines the 32 groups,
-// then one thread per column.  CTAs [col_ctas, ...): one thread per row.
-constexpr int kK2Cols = 8;       // vector columns per CTA
-constexpr int kK2Groups = 32;    // partial-row groups per CTA
-
+// From the partial maxima of pass 1: one block of the scale-vector step (cq_passes.cuh) per CTA.
 template <int DT>
 __global__ void __launch_bounds__(kThreads)
 k2_scales_from_partials(int64_t T, int64_t I, int I8, int nstrips, int Y, int col_ctas,
@@ -178,50 +173,11 @@ k2_scales_from_partials(int64_t T, int64_t I, int I8, int nstrips, int Y, int co
                         float* __restrict__ a, float* __restrict__ b, float* __restrict__ ra, float* __restrict__ rb,
                         unsigned long long* __restrict__ zero_count) {
     __shared__ uint4 s_part[kK2Groups][kK2Cols];
-    const int tid = threadIdx.x;
     asm volatile("griddepcontrol.launch_dependents;");
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (blockIdx.x == 0 && tid == 0 && zero_count != nullptr) *zero_count = 0ull;
-    if (static_cast<int>(blockIdx.x) < col_ctas) {
-        const int vx = tid & (kK2Cols - 1), grp = tid / kK2Cols;
-        const int vcol = blockIdx.x * kK2Cols + vx;
-        uint4 m = make_uint4(0, 0, 0, 0);
-        if (vcol < I8) {
-#pragma unroll 4
-            for (int y = grp; y < Y; y += kK2Groups) {
-                const uint4 w = colpart[static_cast<int64_t>(y) * I8 + vcol];
-                m.x = max_u16x2(m.x, w.x); m.y = max_u16x2(m.y, w.y);
-                m.z = max_u16x2(m.z, w.z); m.w = max_u16x2(m.w, w.w);
-            }
-        }
-        s_part[grp][vx] = m;
-        __syncthreads();
-        const int64_t j = static_cast<int64_t>(blockIdx.x) * (kK2Cols * 8) + tid;
-        if (tid < kK2Cols * 8 && j < I) {
-            const uint16_t* sp = reinterpret_cast<const uint16_t*>(&s_part[0][0]);
-            uint32_t mx = 0;
-#pragma unroll
-            for (int k = 0; k < kK2Groups; ++k) mx = max(mx, static_cast<uint32_t>(sp[k * (kK2Cols * 8) + tid]));
-            const float cj = cvt16<DT>(static_cast<uint16_t>(mx));
-            if (c_out != nullptr) c_out[j] = cj;
-            float bj, rbj;
-            col_scale_of(cj, alpha, qmax, bj, rbj);
-            b[j] = bj;
-            rb[j] = rbj;
-        }
-    } else {
-        const int64_t i = static_cast<int64_t>(blockIdx.x - col_ctas) * kThreads + tid;
-        if (i < T) {
-            uint32_t m = 0;
-            for (int sx = 0; sx < nstrips; ++sx) m = max(m, static_cast<uint32_t>(rowpart[i * nstrips + sx]));
-            const float ti = cvt16<DT>(static_cast<uint16_t>(m));
-            if (t_out != nullptr) t_out[i] = ti;
-            float ai, rai;
-            row_scale_of(ti, alpha, qmax, ai, rai);
-            a[i] = ai;
-            ra[i] = rai;
-        }
-    }
+    if (blockIdx.x == 0 && threadIdx.x == 0 && zero_count != nullptr) *zero_count = 0ull;
+    scales_block<DT>(static_cast<int>(blockIdx.x), T, I, I8, nstrips, Y, col_ctas, rowpart, colpart, alpha, qmax,
+                     t_out, c_out, a, b, ra, rb, s_part);
 }
 
 // From finished t, c (the general path, and callers that supply the absmax vectors): one thread
@@ -293,6 +249,7 @@ k3_quantize(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
     constexpr bool STAGED = MODE != 0;
     extern __shared__ __align__(128) unsigned char s_dyn[];
     __shared__ uint64_t s_full[kStages];
+    __shared__ int s_abort;                      // a wait on a row copy gave up: the CTA stops issuing and leaves
     const int tid = threadIdx.x, lane = tid & 31;
     const int v = blockIdx.x * blockDim.x + tid;
     const bool active = v < I8;
@@ -302,117 +259,84 @@ k3_quantize(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
     const int64_t Y = gridDim.y;
     unsigned int zeros = 0;
 
-    // Everything this kernel reads except X is produced by the preceding kernel of the stream.
+    // ---- staged: ring geometry, barriers and the first copies.  X is an input of the whole call, not a product of
+    // the preceding kernel, so the ring is filled while that kernel (the scale vectors) is still running.
+    uint4* stage = reinterpret_cast<uint4*>(s_dyn);                   // [kStages][4 rows][blockDim.x]
+    const int Wv = blockDim.x;
+    const int strip0 = blockIdx.x * Wv;
+    const uint32_t seg_bytes = static_cast<uint32_t>(min(Wv, I8 - strip0)) * 16u;
+    const int64_t first = blockIdx.y;
+    const int64_t mine = (STAGED && first < nfull) ? (nfull - first + Y - 1) / Y : 0;      // groups of this CTA
+    auto group_at = [&](int64_t k) { const int64_t pos = first + k * Y; return forward ? pos : nfull - 1 - pos; };
+    auto issue = [&](int64_t k) {                                     // thread 0 only
+        if (k >= mine) return;
+        const int st = static_cast<int>(k % kStages);
+        const uint4* src = X + (group_at(k) << 2) * ld8 + strip0;
+        mbar_expect_tx(&s_full[st], 4u * seg_bytes);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) bulk_load(stage + (st * 4 + u) * Wv, src + u * ld8, seg_bytes, &s_full[st]);
+    };
+    if constexpr (STAGED) {
+        if (tid == 0) {
+            s_abort = 0;
+#pragma unroll
+            for (int st = 0; st < kStages; ++st) mbar_init(&s_full[st], 1);
+            mbar_init_fence();
+            for (int k = 0; k < kStages - 1; ++k) issue(k);
+        }
+        __syncthreads();
+    }
+
+    // Everything else this kernel reads is produced by the preceding kernel of the stream.
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
     if (warp_active || STAGED) {
-        float2 b2[4], rb2[4];
-        {
-            const float4* bp = reinterpret_cast<const float4*>(b) + static_cast<int64_t>(vv) * 2;
-            const float4* rp = reinterpret_cast<const float4*>(rb) + static_cast<int64_t>(vv) * 2;
-            const float4 b0 = __ldg(bp), b1 = __ldg(bp + 1), q0 = __ldg(rp), q1 = __ldg(rp + 1);
-            b2[0] = make_float2(b0.x, b0.y); b2[1] = make_float2(b0.z, b0.w);
-            b2[2] = make_float2(b1.x, b1.y); b2[3] = make_float2(b1.z, b1.w);
-            rb2[0] = make_float2(q0.x, q0.y); rb2[1] = make_float2(q0.z, q0.w);
-            rb2[2] = make_float2(q1.x, q1.y); rb2[3] = make_float2(q1.z, q1.w);
-        }
-        // false if any of this thread's eight column reciprocals is the NaN marker of an extreme scale
-        const bool cols_trusted = ((rb2[0].x + rb2[0].y) + (rb2[1].x + rb2[1].y)) +
-                                  ((rb2[2].x + rb2[2].y) + (rb2[3].x + rb2[3].y)) < INFINITY;
+        const ColumnScales cs = load_column_scales(b, rb, vv);
         const uint4* xp = X + vv;
-
-        // One row of 8 elements: quantize, re-load the row slot for the next group, pack, store
-        // (stores only from lanes that own a column).  `vec` indexes 8-element vectors of the outputs.
-        auto do_row = [&](uint4& slot, const uint4* reload, bool has_next, float au, float rau, int vec) {
-            float2 y2[4], q2[4];
-            quantize_row8<DT, BITS, false>(slot, au, rau, b2, rb2, cols_trusted && rau == rau, y2, q2);
-            if (has_next) slot = ld_stream(reload);
-            if constexpr (BITS == 8) {
-                const uint32_t c0 = pack_int8x4(y2[0].x, y2[0].y, y2[1].x, y2[1].y);
-                const uint32_t c1 = pack_int8x4(y2[2].x, y2[2].y, y2[3].x, y2[3].y);
-                if constexpr (COUNT) zeros += zero_bytes(c0) + zero_bytes(c1);
-                if constexpr (CODES) { if (active) st_stream(reinterpret_cast<uint2*>(codes) + vec, make_uint2(c0, c1)); }
-            } else {
-                const uint32_t c0 = pack_int4x8(y2);
-                if constexpr (COUNT) zeros += zero_nibbles(c0);
-                if constexpr (CODES) { if (active) st_stream(reinterpret_cast<uint32_t*>(codes) + vec, c0); }
-            }
-            if constexpr (DEQ != 0) {
-                const float2 a2 = make_float2(au, au);
-                float2 d2[4];
-#pragma unroll
-                for (int k = 0; k < 4; ++k) d2[k] = __fmul2_rn(q2[k], __fmul2_rn(a2, b2[k]));
-                if constexpr (DEQ == 1) {
-                    uint4 o;
-                    o.x = pack16x2<DT>(d2[0].x, d2[0].y); o.y = pack16x2<DT>(d2[1].x, d2[1].y);
-                    o.z = pack16x2<DT>(d2[2].x, d2[2].y); o.w = pack16x2<DT>(d2[3].x, d2[3].y);
-                    if (active) st_stream(reinterpret_cast<uint4*>(deq) + vec, o);
-                } else {
-                    float4* o = reinterpret_cast<float4*>(deq) + static_cast<int64_t>(vec) * 2;
-                    if (active) {
-                        st_stream(o, make_float4(d2[0].x, d2[0].y, d2[1].x, d2[1].y));
-                        st_stream(o + 1, make_float4(d2[2].x, d2[2].y, d2[3].x, d2[3].y));
-                    }
-                }
-            }
-        };
         // lanes 0-3 fetch a_i of a group's four rows, lanes 4-7 the reciprocals (rows clamped to T-1)
         auto load_scales = [&](int64_t g) {
             const int64_t row = min((g << 2) + (lane & 3), T - 1);
             return lane < 8 ? __ldg((lane < 4 ? a : ra) + row) : 0.0f;
+        };
+        auto do_row = [&](const uint4& x, float au, float rau, int vec) {
+            quantize_store_row8<DT, BITS, DEQ, CODES, COUNT>(x, au, rau, cs, active, vec, codes, deq, zeros);
         };
 
         if ((T & 3) != 0 && blockIdx.y == 0 && warp_active) {          // ragged last group
             const float arv = load_scales(nfull);
             for (int u = 0; u < static_cast<int>(T & 3); ++u) {
                 const int64_t row = (nfull << 2) + u;
-                uint4 slot = ld_stream(xp + row * ld8);
-                do_row(slot, nullptr, false, __shfl_sync(0xFFFFFFFFu, arv, u), __shfl_sync(0xFFFFFFFFu, arv, 4 + u),
+                do_row(ld_stream(xp + row * ld8), __shfl_sync(0xFFFFFFFFu, arv, u), __shfl_sync(0xFFFFFFFFu, arv, 4 + u),
                        static_cast<int>(row * I8 + vv));
             }
         }
 
         if constexpr (STAGED) {
-            uint4* stage = reinterpret_cast<uint4*>(s_dyn);               // [kStages][4 rows][blockDim.x]
-            const int Wv = blockDim.x;
-            const int strip0 = blockIdx.x * Wv;
-            const uint32_t seg_bytes = static_cast<uint32_t>(min(Wv, I8 - strip0)) * 16u;
-            const int64_t first = blockIdx.y;
-            const int64_t mine = first < nfull ? (nfull - first + Y - 1) / Y : 0;      // groups of this CTA
-            auto group_at = [&](int64_t k) { const int64_t pos = first + k * Y; return forward ? pos : nfull - 1 - pos; };
-            auto issue = [&](int64_t k) {                                 // thread 0 only
-                if (k >= mine) return;
-                const int st = static_cast<int>(k % kStages);
-                const uint4* src = X + (group_at(k) << 2) * ld8 + strip0;
-                mbar_expect_tx(&s_full[st], 4u * seg_bytes);
-#pragma unroll
-                for (int u = 0; u < 4; ++u) bulk_load(stage + (st * 4 + u) * Wv, src + u * ld8, seg_bytes, &s_full[st]);
-            };
-            if (tid == 0) {
-#pragma unroll
-                for (int st = 0; st < kStages; ++st) mbar_init(&s_full[st], 1);
-                mbar_init_fence();
-            }
-            __syncthreads();
-            if (tid == 0) {
-                for (int k = 0; k < kStages - 1; ++k) issue(k);
-            }
-            for (int64_t k = 0; k < mine; ++k) {
+            int64_t k = 0;
+            for (; k < mine; ++k) {
                 const int64_t g = group_at(k);
                 const float arv = load_scales(g);
                 __syncthreads();                                          // everybody is done with group k-1: its stage is free
+                if (s_abort) break;
                 if (tid == 0) issue(k + kStages - 1);
                 const int st = static_cast<int>(k % kStages);
-                if (!mbar_wait(&s_full[st], static_cast<uint32_t>((k / kStages) & 1))) atomicExch(&g_stage_fault, 1u);
+                if (!mbar_wait(&s_full[st], static_cast<uint32_t>((k / kStages) & 1))) {
+                    atomicExch(&g_stage_fault, 1u);
+                    s_abort = 1;                                          // seen by everybody after the next barrier
+                }
                 if (warp_active) {
                     const int vec = static_cast<int>((g << 2) * I8 + vv);
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        uint4 cur = stage[(st * 4 + u) * Wv + tid];
-                        do_row(cur, nullptr, false, __shfl_sync(0xFFFFFFFFu, arv, u), __shfl_sync(0xFFFFFFFFu, arv, 4 + u),
-                               vec + u * I8);
-                    }
+                    for (int u = 0; u < 4; ++u)
+                        do_row(stage[(st * 4 + u) * Wv + tid], __shfl_sync(0xFFFFFFFFu, arv, u),
+                               __shfl_sync(0xFFFFFFFFu, arv, 4 + u), vec + u * I8);
                 }
+            }
+            if (k < mine && tid == 0) {
+                // Abandoned: nothing more is issued; the copies still in flight (groups k .. k + kStages - 2) get one
+                // more bounded wait each so that none of them lands in shared memory the next CTA already owns.
+                for (int64_t kk = k; kk < min(mine, k + kStages - 1); ++kk)
+                    mbar_wait(&s_full[kk % kStages], static_cast<uint32_t>((kk / kStages) & 1));
             }
         }
 
@@ -434,9 +358,11 @@ k3_quantize(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
                 float arvn = 0.0f;
                 if (has_next) arvn = load_scales(g + dgroups);
 #pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    do_row(w[u], pn + u * ld8, has_next, __shfl_sync(0xFFFFFFFFu, arv, u),
-                           __shfl_sync(0xFFFFFFFFu, arv, 4 + u), vec + u * I8);
+                for (int u = 0; u < 4; ++u) {
+                    const uint4 cur = w[u];
+                    if (has_next) w[u] = ld_stream(pn + u * ld8);
+                    do_row(cur, __shfl_sync(0xFFFFFFFFu, arv, u), __shfl_sync(0xFFFFFFFFu, arv, 4 + u), vec + u * I8);
+                }
                 p = pn;
                 vec += ostep;
                 g += dgroups;
@@ -491,6 +417,9 @@ static int g_tune_k3_forward = 0;   // walk pass 2 in ascending row order
 static int g_tune_no_pdl = 0;       // launch pass 2 without programmatic dependent launch
 static int g_tune_no_small = 0;     // never take the single-launch path for small matrices
 static int g_tune_no_stage = 0;     // pass 2 loads rows straight into registers instead of staging them
+static int g_tune_no_fused = 0;     // never take the single cooperative launch for on-chip-sized matrices
+static int g_tune_fused_max_mb = 0; // largest X (MB) that takes it (0 = the built-in limit)
+constexpr int kFusedMaxMB = 128;
 static cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
 
 static inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
@@ -530,7 +459,9 @@ Plan make_plan(int64_t T, int64_t I) {
     p.off_rb = carve(sizeof(float) * static_cast<size_t>(p.I8) * 8);
     p.off_rowpart = carve(sizeof(uint16_t) * static_cast<size_t>(T) * p.nstrips);
     const int64_t ymax = p.ngroups < p.ycap ? (p.ngroups > 0 ? p.ngroups : 1) : p.ycap;
+    p.ymax = ymax;
     p.off_colpart = carve(sizeof(uint16_t) * static_cast<size_t>(ymax) * static_cast<size_t>(p.I8) * 8);
+    p.off_sync = carve(kFusedSyncBytes);
     return p;
 }
 
@@ -774,6 +705,25 @@ int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
         }
     }
 
+    // ---- matrices the chip can hold: one cooperative launch (the timing hook needs the quantize pass as a kernel of its own)
+    if (!given && fast_in && fast_out && !g_tune_no_fused && (g_ev_before == nullptr || g_ev_after == nullptr) &&
+        (codes != nullptr || deq != nullptr || zero_count != nullptr) &&
+        T * ld * 2 <= static_cast<int64_t>(g_tune_fused_max_mb > 0 ? g_tune_fused_max_mb : kFusedMaxMB) << 20) {
+        const FusedArgs fa{X, dtype, T, I, p.I8, ld / 8, p.W, p.nstrips, p.ymax, alpha, bits, rowpart, colpart,
+                           t_dev, c_dev, a_dev, b_dev, ra_dev, rb_dev,
+                           codes, deq, deq == nullptr ? 0 : (deq_dtype == CQ_F32 ? 2 : 1), zero_count, ws + p.off_sync};
+        if (launch_fused(fa, st)) {
+            if ((rc = launch_status()) != CQ_OK) return rc;
+            if (c != nullptr && !c_in_place &&
+                cudaMemcpyAsync(c, c_dev, sizeof(float) * I, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+                return CQ_ERR_CUDA;
+            if (col_scale != nullptr && !b_in_place &&
+                cudaMemcpyAsync(col_scale, b_dev, sizeof(float) * I, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+                return CQ_ERR_CUDA;
+            return CQ_OK;
+        }
+    }
+
     // ---- pass 1 + scale vectors
     if (given) {
         k2_scales_from_vectors<<<k2v_blocks, kThreads, 0, st>>>(T, I, t_given, c_given, alpha, qmax, a_dev, b_dev,
@@ -865,9 +815,11 @@ const char* cq_status_string(int status) {
 
 int cq_set_tuning(const char* key, int value) {
     if (key == nullptr) return CQ_ERR_NULL;
-    if (value > 64) return CQ_ERR_SHAPE;
     auto eq = [](const char* x, const char* y) { while (*x && *x == *y) { ++x; ++y; } return *x == *y; };
     const int v = value > 0 ? value : 0;
+    if (eq(key, "fused_max_mb")) { if (v > (1 << 20)) return CQ_ERR_SHAPE; cq::g_tune_fused_max_mb = v; return CQ_OK; }
+    if (v > 64) return CQ_ERR_SHAPE;
+    if (eq(key, "no_fused")) { cq::g_tune_no_fused = v ? 1 : 0; return CQ_OK; }
     if (eq(key, "k1_ctas_per_sm")) { cq::g_tune_k1_ctas = v; return CQ_OK; }
     if (eq(key, "k3_ctas_per_sm")) { cq::g_tune_k3_ctas = v; return CQ_OK; }
     if (eq(key, "k3_forward")) { cq::g_tune_k3_forward = v ? 1 : 0; return CQ_OK; }
@@ -879,13 +831,14 @@ int cq_set_tuning(const char* key, int value) {
 
 int cq_stage_fault(unsigned int* fault_host) {
     if (fault_host == nullptr) return CQ_ERR_NULL;
-    unsigned int quantize_pass = 0, diagnostics = 0, weights = 0, small = 0;
+    unsigned int quantize_pass = 0, diagnostics = 0, weights = 0, small = 0, fused = 0;
     if (cudaMemcpyFromSymbol(&quantize_pass, cq::g_stage_fault, sizeof(unsigned int)) != cudaSuccess) return CQ_ERR_CUDA;
     int rc = cq::diag_stage_fault(&diagnostics);
     if (rc == CQ_OK) rc = cq::weight_stage_fault(&weights);
     if (rc == CQ_OK) rc = cq::small_stage_fault(&small);
+    if (rc == CQ_OK) rc = cq::fused_fault(&fused);
     if (rc != CQ_OK) return rc;
-    *fault_host = quantize_pass | diagnostics | weights | small;
+    *fault_host = quantize_pass | diagnostics | weights | small | fused;
     return CQ_OK;
 }
 

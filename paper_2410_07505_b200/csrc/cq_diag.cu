@@ -70,6 +70,33 @@ k9_zero_tests(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
     unsigned int n_removed = 0, n_pt = 0, n_cq = 0;
     extern __shared__ __align__(128) unsigned char s_dyn[];
     __shared__ uint64_t s_full[kRing];
+    __shared__ int s_abort;                      // a wait on a row copy gave up: the CTA stops issuing and leaves
+
+    // Ring geometry, barriers and the first copies: X is an input of the call, not a product of the preceding
+    // kernel (the scale vectors), so the ring fills while that kernel is still running.
+    uint4* stage = reinterpret_cast<uint4*>(s_dyn);                   // [kRing][4 rows][blockDim.x]
+    const int Wv = blockDim.x;
+    const int strip0 = blockIdx.x * Wv;
+    const uint32_t seg_bytes = static_cast<uint32_t>(min(Wv, I8 - strip0)) * 16u;
+    const int64_t first = blockIdx.y;
+    const int64_t mine = first < nfull ? (nfull - first + Y - 1) / Y : 0;          // groups of this CTA
+    auto group_at = [&](int64_t k) { return nfull - 1 - (first + k * Y); };
+    auto issue = [&](int64_t k) {                                     // thread 0 only
+        if (k >= mine) return;
+        const int st = static_cast<int>(k % kRing);
+        const uint4* src = X + (group_at(k) << 2) * ld8 + strip0;
+        mbar_expect_tx(&s_full[st], 4u * seg_bytes);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) bulk_load(stage + (st * 4 + u) * Wv, src + u * ld8, seg_bytes, &s_full[st]);
+    };
+    if (tid == 0) {
+        s_abort = 0;
+#pragma unroll
+        for (int st = 0; st < kRing; ++st) mbar_init(&s_full[st], 1);
+        mbar_init_fence();
+        for (int k = 0; k < kRing - 1; ++k) issue(k);
+    }
+    __syncthreads();
 
     // the scale vectors come from the preceding kernel of the stream
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -186,39 +213,20 @@ k9_zero_tests(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
             }
         }
 
-        uint4* stage = reinterpret_cast<uint4*>(s_dyn);                   // [kRing][4 rows][blockDim.x]
-        const int Wv = blockDim.x;
-        const int strip0 = blockIdx.x * Wv;
-        const uint32_t seg_bytes = static_cast<uint32_t>(min(Wv, I8 - strip0)) * 16u;
-        const int64_t first = blockIdx.y;
-        const int64_t mine = first < nfull ? (nfull - first + Y - 1) / Y : 0;          // groups of this CTA
-        auto group_at = [&](int64_t k) { return nfull - 1 - (first + k * Y); };
-        auto issue = [&](int64_t k) {                                     // thread 0 only
-            if (k >= mine) return;
-            const int st = static_cast<int>(k % kRing);
-            const uint4* src = X + (group_at(k) << 2) * ld8 + strip0;
-            mbar_expect_tx(&s_full[st], 4u * seg_bytes);
-#pragma unroll
-            for (int u = 0; u < 4; ++u) bulk_load(stage + (st * 4 + u) * Wv, src + u * ld8, seg_bytes, &s_full[st]);
-        };
-        if (tid == 0) {
-#pragma unroll
-            for (int st = 0; st < kRing; ++st) mbar_init(&s_full[st], 1);
-            mbar_init_fence();
-        }
-        __syncthreads();
-        if (tid == 0) {
-            for (int k = 0; k < kRing - 1; ++k) issue(k);
-        }
         float raw = mine > 0 ? load_scale(group_at(0)) : 0.0f;
-        for (int64_t k = 0; k < mine; ++k) {
+        int64_t k = 0;
+        for (; k < mine; ++k) {
             const int64_t g = group_at(k);
             const float tv = threshold_of(raw);
             if (k + 1 < mine) raw = load_scale(group_at(k + 1));
             __syncthreads();                                              // everybody is done with group k-1: its stage is free
+            if (s_abort) break;
             if (tid == 0) issue(k + kRing - 1);
             const int st = static_cast<int>(k % kRing);
-            if (!mbar_wait(&s_full[st], static_cast<uint32_t>((k / kRing) & 1))) atomicExch(&g_diag_stage_fault, 1u);
+            if (!mbar_wait(&s_full[st], static_cast<uint32_t>((k / kRing) & 1))) {
+                atomicExch(&g_diag_stage_fault, 1u);
+                s_abort = 1;                                              // seen by everybody after the next barrier
+            }
             if (warp_active) {
                 const int vec = static_cast<int>((g << 2) * I8 + vv);
 #pragma unroll
@@ -229,6 +237,11 @@ k9_zero_tests(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
                     do_row(cur, thr, (g << 2) + u, vec + u * I8);
                 }
             }
+        }
+        if (k < mine && tid == 0) {
+            // abandoned: nothing more is issued; one more bounded wait for each copy still in flight
+            for (int64_t kk = k; kk < min(mine, k + kRing - 1); ++kk)
+                mbar_wait(&s_full[kk % kRing], static_cast<uint32_t>((kk / kRing) & 1));
         }
         if (!active) { n_removed = 0; n_pt = 0; n_cq = 0; }
     }
