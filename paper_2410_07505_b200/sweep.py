@@ -124,11 +124,16 @@ def main() -> None:
     ap.add_argument("--alpha", type=float, default=0.15)
     ap.add_argument("--decode", action="store_true", help="time decode-sized matrices through the single-launch path, "
                     "the three launches and a CUDA-graph replay, then exit")
+    ap.add_argument("--tune", action="append", default=[], metavar="KEY=VALUE",
+                    help="launch-shape knob to set before timing (see cq_set_tuning), e.g. no_fused=1; may be repeated")
     ap.add_argument("--only", default="", help="comma-separated config names (e.g. llama70b_mlp,weight_8192x28672): "
                     "time only these (keeps a profiler capture short)")
     args = ap.parse_args()
     only = set(filter(None, args.only.split(",")))
     cq.lib()
+    for kv in args.tune:
+        key, _, value = kv.partition("=")
+        cq.set_tuning(key, int(value))
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     if args.decode:
         time_decode_shapes(flush, args.iters)

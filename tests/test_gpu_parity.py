@@ -211,6 +211,7 @@ def test_public_call_replays_from_a_cuda_graph(cq, shape):
             b.zero_()
         graph.replay()
         torch.cuda.synchronize()
+        buf.arena.check("graph replay")
         parity.check_act(X, "bf16", 0.15, 8, t=buf.t.cpu().numpy(), c=buf.c.cpu().numpy(), a=buf.row_scale.cpu().numpy(),
                          b=buf.col_scale.cpu().numpy(), codes=buf.codes.cpu().numpy(), deq=bits_of(buf.deq),
                          zero_count=int(buf.zero_count.item()))
