@@ -21,7 +21,6 @@ import json
 import os
 import statistics
 import sys
-import threading
 import time
 
 import numpy as np
@@ -38,7 +37,7 @@ BYTES_PER_ELEMENT_STEP = 7.0        # X read twice (2+2) + int8 codes (1) + bf16
 BYTES_PER_ELEMENT_QUANT_PASS = 5.0  # quantize pass alone: X (2) + codes (1) + dequantized (2)
 FALLBACK_HBM_GBS = 6650.0
 L2_FLUSH_BYTES = 256 << 20
-HOOK_EVERY = 8
+HOOK_LAUNCHES = 64          # launches of the quantize pass timed inside real calls for the roofline object
 
 # DRAM traffic of the quantize pass from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum
 # per launch), valid only for the kernel sources whose digest is recorded with it.
@@ -62,60 +61,6 @@ def measured_peak():
             return float(json.load(f)["hbm_gbs"]), "measured"
     except Exception:
         return FALLBACK_HBM_GBS, "fallback"
-
-
-class ClockSampler:
-    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
-
-    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
-               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown"}
-
-    def __init__(self, index: int, uuid: str | None = None, period_s: float = 0.02):
-        self.index, self.period = index, period_s
-        self.samples, self.reasons, self.max_mhz = [], set(), None
-        self._stop = threading.Event()
-        self._thread = None
-        try:
-            import pynvml
-            pynvml.nvmlInit()
-            self.nvml = pynvml
-            try:
-                self.handle = pynvml.nvmlDeviceGetHandleByUUID(f"GPU-{uuid}".encode() if uuid else b"")
-            except Exception:
-                self.handle = pynvml.nvmlDeviceGetHandleByIndex(index)
-            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
-        except Exception:
-            self.nvml = None
-
-    def _run(self):
-        n = self.nvml
-        while not self._stop.is_set():
-            try:
-                self.samples.append(int(n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM)))
-                mask = int(n.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
-                for bit, name in self.REASONS.items():
-                    if mask & bit:
-                        self.reasons.add(name)
-            except Exception:
-                pass
-            self._stop.wait(self.period)
-
-    def __enter__(self):
-        if self.nvml is not None:
-            self._thread = threading.Thread(target=self._run, daemon=True)
-            self._thread.start()
-        return self
-
-    def __exit__(self, *exc):
-        self._stop.set()
-        if self._thread is not None:
-            self._thread.join()
-
-    def summary(self):
-        if not self.samples:
-            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
-        return {"sm_mhz": int(statistics.median(self.samples)), "sm_max_mhz": self.max_mhz,
-                "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
 def rank_config(rank: int):
@@ -192,7 +137,7 @@ def main() -> None:
     import torch
     import torch.distributed as dist
 
-    from paper_2410_07505_b200 import build as cuda_build, cq, workloads as wl
+    from paper_2410_07505_b200 import build as cuda_build, clocks as clk, cq, workloads as wl
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -213,46 +158,60 @@ def main() -> None:
     Xh = torch.from_numpy(X.view(np.int16)).view(torch.bfloat16)
     Xd = Xh.cuda()
     buf = cq.ActBuffers(T, I, torch.bfloat16, BITS)
-    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda").zero_()
+    flush_words = flush.view(torch.int32)
+    flush_sum = torch.zeros((), dtype=torch.int64, device="cuda")
+
+    def flush_l2(kind: str) -> None:
+        """Untimed, between steps.  "read": a 256 MiB read pushes X and the outputs out of L2 and leaves clean lines
+        behind.  "write": a 256 MiB fill does the same but leaves 126 MB of dirty lines, whose write-back then
+        competes with the step's first pass (reported beside the headline, not as it)."""
+        if kind == "read":
+            torch.sum(flush_words, dim=0, out=flush_sum)
+        elif kind == "write":
+            flush.zero_()
 
     def step():
         cq.quantize_act(Xd, ALPHA, BITS, buffers=buf)
 
     for _ in range(args.warmup):
-        flush.zero_()
+        flush_l2("read")
         step()
     torch.cuda.synchronize()
 
     K = args.steps
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
-    # The quantize pass is timed inside the real call on every HOOK_EVERY-th step only: the two extra
-    # event records sit between dependent kernels and cost a few microseconds of overlap.
-    hooked = [k for k in range(K) if k % HOOK_EVERY == 0]
-    for k in hooked:                               # torch creates the CUDA event on first record
-        ev[k][2].record()
-        ev[k][3].record()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(K)]
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
-    with ClockSampler(local, str(torch.cuda.get_device_properties(local).uuid)) as clocks:
+    with clk.ClockSampler(local, str(torch.cuda.get_device_properties(local).uuid), period_s=0.002) as clocks:
         for k in range(K):
-            flush.zero_()                         # untimed: evicts X and the outputs from L2
-            if k % HOOK_EVERY == 0:
-                cq.set_timing_events(ev[k][2], ev[k][3])
-            elif k % HOOK_EVERY == 1:
-                cq.set_timing_events(None, None)
+            flush_l2("read")                      # untimed: evicts X and the outputs from L2
             ev[k][0].record()
             step()
             ev[k][1].record()
         torch.cuda.synchronize()
-    cq.set_timing_events(None, None)
     if world > 1:
         dist.barrier()
     step_ms = [e[0].elapsed_time(e[1]) for e in ev]
-    quant_ms = [ev[k][2].elapsed_time(ev[k][3]) for k in hooked]
     total_ms = max_over_ranks(sum(step_ms), "cuda")
     value = whole_job_gbs(n, K, world, total_ms)
     zero_count = int(buf.zero_count.item())
+
+    # ---- the dominant kernel (the quantize pass) timed inside real calls, outside the headline loop: the two extra
+    # event records sit between dependent kernels and cost the call a few microseconds of overlap
+    hook = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(HOOK_LAUNCHES)]
+    for a_, b_ in hook:                              # torch creates the CUDA event on first record
+        a_.record()
+        b_.record()
+    torch.cuda.synchronize()
+    for a_, b_ in hook:
+        flush_l2("read")
+        cq.set_timing_events(a_, b_)
+        step()
+    torch.cuda.synchronize()
+    cq.set_timing_events(None, None)
+    quant_ms = [a_.elapsed_time(b_) for a_, b_ in hook]
 
     # ---- end to end: host buffers in, host buffers out, through cq_quantize_act_host.
     # (a) one call after the other on one stream; (b) the same calls issued alternately on two streams with
@@ -303,7 +262,7 @@ def main() -> None:
             fn()
         for a_, b_ in evs:
             if flushed:
-                flush.zero_()
+                flush_l2(flushed if isinstance(flushed, str) else "read")
             a_.record()
             fn()
             b_.record()
@@ -315,6 +274,10 @@ def main() -> None:
         ms4 = timed(lambda: cq.quantize_act(Xd, ALPHA, 4, buffers=buf4))
         also["act_int4"] = {"ms_per_step": ms4, "gbs": 6.5 * n / (ms4 * 1e-3) / 1e9, "bytes_per_element": 6.5}
         del buf4
+        msw8 = timed(lambda: cq.quantize_act(Xd, ALPHA, BITS, buffers=buf), flushed="write")
+        also["act_int8_after_a_write_flush"] = {
+            "ms_per_step": msw8, "gbs": BYTES_PER_ELEMENT_STEP * n / (msw8 * 1e-3) / 1e9,
+            "l2": "flushed by a 256 MiB fill: the write-back of its 126 MB of dirty lines overlaps the absmax pass"}
         ms8 = timed(lambda: cq.quantize_act(Xd, ALPHA, BITS, buffers=buf), flushed=False)
         also["act_int8_back_to_back"] = {"ms_per_step": ms8, "gbs": BYTES_PER_ELEMENT_STEP * n / (ms8 * 1e-3) / 1e9,
                                          "l2": "not flushed: X (235 MB) and the outputs (352 MB) exceed the 126 MB L2"}
@@ -340,7 +303,8 @@ def main() -> None:
         "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": workload_name(cfg),
-                   "l2": "flushed between steps (256 MiB write, untimed); X (235 MB) also exceeds the 126 MB L2",
+                   "l2": "flushed between steps by an untimed 256 MiB read (clean lines); X (235 MB) also exceeds the "
+                         "126 MB L2; the same step after a 256 MiB write flush and back to back: see also",
                    "timing": "CUDA events per step on the launch stream, summed; max over ranks",
                    "bytes_per_element": BYTES_PER_ELEMENT_STEP, "per_rank": "independent matrices, no collective"},
         "elements_per_s": n * K * world / (total_ms * 1e-3),
@@ -359,7 +323,7 @@ def main() -> None:
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": f"of {peak_kind}", "traffic": traffic,
                      "algorithmic_bytes_per_launch": BYTES_PER_ELEMENT_QUANT_PASS * n,
-                     "avg_launch_ms": quant_mean_ms, "launches_timed": len(hooked)},
+                     "avg_launch_ms": quant_mean_ms, "launches_timed": len(quant_ms)},
     }
 
     # ---- the oracle on the host cores, bounded sample of the same workload

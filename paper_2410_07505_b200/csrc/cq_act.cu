@@ -417,9 +417,6 @@ static int g_tune_k3_forward = 0;   // walk pass 2 in ascending row order
 static int g_tune_no_pdl = 0;       // launch pass 2 without programmatic dependent launch
 static int g_tune_no_small = 0;     // never take the single-launch path for small matrices
 static int g_tune_no_stage = 0;     // pass 2 loads rows straight into registers instead of staging them
-static int g_tune_no_fused = 0;     // never take the single cooperative launch for on-chip-sized matrices
-static int g_tune_fused_max_mb = 0; // largest X (MB) that takes it (0 = the built-in limit)
-constexpr int kFusedMaxMB = 128;
 static cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
 
 static inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
@@ -459,9 +456,7 @@ Plan make_plan(int64_t T, int64_t I) {
     p.off_rb = carve(sizeof(float) * static_cast<size_t>(p.I8) * 8);
     p.off_rowpart = carve(sizeof(uint16_t) * static_cast<size_t>(T) * p.nstrips);
     const int64_t ymax = p.ngroups < p.ycap ? (p.ngroups > 0 ? p.ngroups : 1) : p.ycap;
-    p.ymax = ymax;
     p.off_colpart = carve(sizeof(uint16_t) * static_cast<size_t>(ymax) * static_cast<size_t>(p.I8) * 8);
-    p.off_sync = carve(kFusedSyncBytes);
     return p;
 }
 
@@ -705,25 +700,6 @@ int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
         }
     }
 
-    // ---- matrices the chip can hold: one cooperative launch (the timing hook needs the quantize pass as a kernel of its own)
-    if (!given && fast_in && fast_out && !g_tune_no_fused && (g_ev_before == nullptr || g_ev_after == nullptr) &&
-        (codes != nullptr || deq != nullptr || zero_count != nullptr) &&
-        T * ld * 2 <= static_cast<int64_t>(g_tune_fused_max_mb > 0 ? g_tune_fused_max_mb : kFusedMaxMB) << 20) {
-        const FusedArgs fa{X, dtype, T, I, p.I8, ld / 8, p.W, p.nstrips, p.ymax, alpha, bits, rowpart, colpart,
-                           t_dev, c_dev, a_dev, b_dev, ra_dev, rb_dev,
-                           codes, deq, deq == nullptr ? 0 : (deq_dtype == CQ_F32 ? 2 : 1), zero_count, ws + p.off_sync};
-        if (launch_fused(fa, st)) {
-            if ((rc = launch_status()) != CQ_OK) return rc;
-            if (c != nullptr && !c_in_place &&
-                cudaMemcpyAsync(c, c_dev, sizeof(float) * I, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
-                return CQ_ERR_CUDA;
-            if (col_scale != nullptr && !b_in_place &&
-                cudaMemcpyAsync(col_scale, b_dev, sizeof(float) * I, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
-                return CQ_ERR_CUDA;
-            return CQ_OK;
-        }
-    }
-
     // ---- pass 1 + scale vectors
     if (given) {
         k2_scales_from_vectors<<<k2v_blocks, kThreads, 0, st>>>(T, I, t_given, c_given, alpha, qmax, a_dev, b_dev,
@@ -817,9 +793,7 @@ int cq_set_tuning(const char* key, int value) {
     if (key == nullptr) return CQ_ERR_NULL;
     auto eq = [](const char* x, const char* y) { while (*x && *x == *y) { ++x; ++y; } return *x == *y; };
     const int v = value > 0 ? value : 0;
-    if (eq(key, "fused_max_mb")) { if (v > (1 << 20)) return CQ_ERR_SHAPE; cq::g_tune_fused_max_mb = v; return CQ_OK; }
     if (v > 64) return CQ_ERR_SHAPE;
-    if (eq(key, "no_fused")) { cq::g_tune_no_fused = v ? 1 : 0; return CQ_OK; }
     if (eq(key, "k1_ctas_per_sm")) { cq::g_tune_k1_ctas = v; return CQ_OK; }
     if (eq(key, "k3_ctas_per_sm")) { cq::g_tune_k3_ctas = v; return CQ_OK; }
     if (eq(key, "k3_forward")) { cq::g_tune_k3_forward = v ? 1 : 0; return CQ_OK; }
@@ -831,14 +805,13 @@ int cq_set_tuning(const char* key, int value) {
 
 int cq_stage_fault(unsigned int* fault_host) {
     if (fault_host == nullptr) return CQ_ERR_NULL;
-    unsigned int quantize_pass = 0, diagnostics = 0, weights = 0, small = 0, fused = 0;
+    unsigned int quantize_pass = 0, diagnostics = 0, weights = 0, small = 0;
     if (cudaMemcpyFromSymbol(&quantize_pass, cq::g_stage_fault, sizeof(unsigned int)) != cudaSuccess) return CQ_ERR_CUDA;
     int rc = cq::diag_stage_fault(&diagnostics);
     if (rc == CQ_OK) rc = cq::weight_stage_fault(&weights);
     if (rc == CQ_OK) rc = cq::small_stage_fault(&small);
-    if (rc == CQ_OK) rc = cq::fused_fault(&fused);
     if (rc != CQ_OK) return rc;
-    *fault_host = quantize_pass | diagnostics | weights | small | fused;
+    *fault_host = quantize_pass | diagnostics | weights | small;
     return CQ_OK;
 }
 

@@ -163,15 +163,6 @@ __device__ __forceinline__ float guarded_rcp(float f) {
     if (f == 0.0f) return 0.0f;
     return (f >= kScaleLo && f <= kScaleHi) ? __fdiv_rn(1.0f, f) : __int_as_float(0x7FC00000);
 }
-// Same contract from the hardware's approximate reciprocal (relative error at most 2^-23 on normal
-// inputs): for kernels that need one reciprocal per small group, where the exact one would dominate.
-// The candidate built from it is x * r with two roundings, 3 * 2^-24 in all: inside the bound below.
-__device__ __forceinline__ float guarded_rcp_approx(float f) {
-    if (f == 0.0f) return 0.0f;
-    float r;
-    asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(f));
-    return (f >= kScaleLo && f <= kScaleHi) ? r : __int_as_float(0x7FC00000);
-}
 // ---- scale factors -------------------------------------------------------------------------
 //   a_i = fl32(pow(t_i, alpha) / qmax), b_j = fl32(pow(c_j, 1 - alpha)) in fp64, with alpha in {0, 1}
 //   special-cased so that they reduce exactly to per-column / per-token quantization, plus the
@@ -199,10 +190,11 @@ __device__ __forceinline__ void col_scale_of(float cj, double alpha, int qmax, f
 constexpr float kAcceptBelow = 0.49993896484375f;       // 1/2 - 2^-14
 
 // Packed fp32x2 arithmetic (bit-identical to the scalar IEEE operations, half the issue slots).
-// y2[k] = kMagic + q and q2[k] = q for elements 2k, 2k+1.  UNIFORM: one scale `a` for the whole row
-// (b2, rb2 unused).  `trusted`: none of the reciprocals involved is the NaN marker (a NaN would not
+// y2[k] = kMagic + q and q2[k] = q for elements 2k, 2k+1; element e has the scale a * b2[e] (per-element scales:
+// the activation path; rows under one scale take exact_codes_uniform_row8 below instead).
+// `trusted`: none of the reciprocals involved is the NaN marker (a NaN would not
 // survive the max below, so it has to be tested where the reciprocals are loaded).
-template <int DT, int BITS, bool UNIFORM, bool LEAN = false>
+template <int DT, int BITS, bool LEAN = false>
 __device__ __forceinline__ void quantize_row8(const uint4& w, float a, float ra, const float2 (&b2)[4],
                                               const float2 (&rb2)[4], bool trusted,
                                               float2 (&y2)[4], float2 (&q2)[4]) {
@@ -215,7 +207,7 @@ __device__ __forceinline__ void quantize_row8(const uint4& w, float a, float ra,
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
         const float2 x = unpack16x2<DT>(words[k]);
-        const float2 r = UNIFORM ? ra2 : __fmul2_rn(ra2, rb2[k]);
+        const float2 r = __fmul2_rn(ra2, rb2[k]);
         const float2 v = __fmul2_rn(x, r);                    // x / s, approximately
         y2[k] = __fadd2_rn(v, m2);
         q2[k] = __fadd2_rn(y2[k], nm2);                       // round-half-even(v), exact
@@ -232,18 +224,18 @@ __device__ __forceinline__ void quantize_row8(const uint4& w, float a, float ra,
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             const float2 x = unpack16x2<DT>(words[k]);
-            const float2 r = UNIFORM ? ra2 : __fmul2_rn(ra2, rb2[k]);
+            const float2 r = __fmul2_rn(ra2, rb2[k]);
             if constexpr (!LEAN) {
                 const float2 f = __ffma2_rn(q2[k], neg1, __fmul2_rn(x, r));
                 if (trusted && fmaxf(fabsf(f.x), fabsf(f.y)) < kAcceptBelow) continue;
             }
             const float xs[2] = {x.x, x.y};
-            const float bs[2] = {UNIFORM ? 1.0f : b2[k].x, UNIFORM ? 1.0f : b2[k].y};
+            const float bs[2] = {b2[k].x, b2[k].y};
             const float rs[2] = {r.x, r.y};
             float ys[2];
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                const float sh = UNIFORM ? a : __fmul_rn(a, bs[h]);
+                const float sh = __fmul_rn(a, bs[h]);
                 bool good;
                 float e;
                 ys[h] = quant_candidate(xs[h], sh, rs[h], qmaxf, good, e);
@@ -252,6 +244,44 @@ __device__ __forceinline__ void quantize_row8(const uint4& w, float a, float ra,
             y2[k] = make_float2(ys[0], ys[1]);
             q2[k] = __fadd2_rn(y2[k], nm2);
         }
+    }
+}
+
+// ---- eight elements under ONE scale (a weight row or group): exact quotients, no test ----------
+// With one scale s per row the correctly rounded reciprocal rs = fl32(1 / s) costs one division per row, and
+// then   q0 = fl32(x rs),  r = x - q0 s  (one FMA, exact),  u = fl32(q0 + r rs)  (one FMA)
+// is the correctly rounded quotient fl32(x / s) itself (the classical residual-corrected division; for this use
+// it is not taken on faith: tests/test_exact_quotient_cpu.py checks it against the IEEE division for every pair
+// of mantissas of up to 11 bits, i.e. every fp16 / bf16 element against every scale fl32(max / qmax) a 16-bit
+// maximum can give, which is exhaustive because binary scaling changes nothing while all values stay normal).
+// The magic-number add then rounds u half to even exactly as the defining sequence does, ties included, so no
+// candidate has to be examined afterwards.  Valid for s in [2^-40, 2^40] (guarded_rcp marks anything else with a
+// NaN, and the caller takes exact_codes_uniform_slow); s == 0 gives rs = 0 and codes 0.  No clamp is needed:
+// |x| <= max and s >= (max / qmax)(1 - 2^-24) keep |u| <= qmax (1 + 2^-23), which rounds to qmax.
+template <int DT>
+__device__ __forceinline__ void exact_codes_uniform_row8(const uint4& w, float s, float rs, float2 (&y2)[4]) {
+    const float2 rs2 = make_float2(rs, rs), ns2 = make_float2(-s, -s), m2 = make_float2(kMagic, kMagic);
+    const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const float2 x = unpack16x2<DT>(words[k]);
+        const float2 q0 = __fmul2_rn(x, rs2);
+        const float2 r = __ffma2_rn(q0, ns2, x);
+        y2[k] = __fadd2_rn(__ffma2_rn(r, rs2, q0), m2);
+    }
+}
+
+// The same codes by the defining sequence, element by element (scales outside [2^-40, 2^40]).  Only scalars cross
+// the out-of-line calls, so the arrays of the caller stay in registers.
+template <int DT, int BITS>
+__device__ __forceinline__ void exact_codes_uniform_slow(const uint4& w, float s, float2 (&y2)[4]) {
+    constexpr float qmaxf = static_cast<float>((1 << (BITS - 1)) - 1);
+    const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const float2 x = unpack16x2<DT>(words[k]);
+        const float y0 = quant_exact(x.x, s, qmaxf), y1 = quant_exact(x.y, s, qmaxf);
+        y2[k] = make_float2(y0, y1);
     }
 }
 

@@ -25,7 +25,6 @@ k7_weight_groups(const uint4* __restrict__ W, int64_t nvec, int C8, int64_t ld8,
     constexpr float qmaxf = static_cast<float>((1 << (BITS - 1)) - 1);
     const int lane = threadIdx.x & 31;
     const int64_t base = (static_cast<int64_t>(blockIdx.x) * kVecPerThread) * kThreads + threadIdx.x;
-    const float2 ones[4] = {make_float2(1.0f, 1.0f), make_float2(1.0f, 1.0f), make_float2(1.0f, 1.0f), make_float2(1.0f, 1.0f)};
     const bool contiguous = ld8 == C8;
     uint4 w[kVecPerThread];
 #pragma unroll
@@ -56,7 +55,7 @@ k7_weight_groups(const uint4* __restrict__ W, int64_t nvec, int C8, int64_t ld8,
             if (lane / G == k) mine = mk;
         }
         const float d = __fdiv_rn(cvt16<DT>(static_cast<uint16_t>(mine)), qmaxf);
-        const float rd = guarded_rcp_approx(d);
+        const float rd = guarded_rcp(d);                             // correctly rounded: the quotients below rely on it
 #pragma unroll
         for (int k = 0; k < kVecPerThread; ++k) {
             dk[k] = __shfl_sync(0xFFFFFFFFu, d, k * G + lane / LANES);
@@ -66,18 +65,30 @@ k7_weight_groups(const uint4* __restrict__ W, int64_t nvec, int C8, int64_t ld8,
 #pragma unroll
         for (int k = 0; k < kVecPerThread; ++k) {
             dk[k] = __fdiv_rn(cvt16<DT>(static_cast<uint16_t>(m16[k])), qmaxf);
-            rdk[k] = guarded_rcp_approx(dk[k]);
+            rdk[k] = guarded_rcp(dk[k]);
         }
+    }
+    // codes of all the thread's vectors: exact quotients in straight-line packed arithmetic; a group whose scale is
+    // outside the range that covers (NaN marker in rdk) sends the thread's vectors to the defining sequence instead
+    float2 y[kVecPerThread][4];
+    bool scales_ok = true;
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) scales_ok = scales_ok && rdk[k] == rdk[k];
+    if (scales_ok) {
+#pragma unroll
+        for (int k = 0; k < kVecPerThread; ++k) exact_codes_uniform_row8<DT>(w[k], dk[k], rdk[k], y[k]);
+    } else {
+#pragma unroll
+        for (int k = 0; k < kVecPerThread; ++k) exact_codes_uniform_slow<DT, BITS>(w[k], dk[k], y[k]);
     }
     unsigned int zeros = 0;
 #pragma unroll
     for (int k = 0; k < kVecPerThread; ++k) {
         const int64_t idx = base + static_cast<int64_t>(k) * kThreads;
-        const float d = dk[k], rd = rdk[k];
+        const float d = dk[k];
         if (idx < nvec) {
             if (scale != nullptr && (idx % LANES) == 0) scale[idx / LANES] = d;
-            float2 y2[4], q2[4];
-            quantize_row8<DT, BITS, true>(w[k], d, rd, ones, ones, rd == rd, y2, q2);
+            const float2 (&y2)[4] = y[k];
             if constexpr (BITS == 8) {
                 const uint32_t c0 = pack_int8x4(y2[0].x, y2[0].y, y2[1].x, y2[1].y);
                 const uint32_t c1 = pack_int8x4(y2[2].x, y2[2].y, y2[3].x, y2[3].y);
@@ -89,10 +100,10 @@ k7_weight_groups(const uint4* __restrict__ W, int64_t nvec, int C8, int64_t ld8,
                 if constexpr (CODES) st_stream(reinterpret_cast<uint32_t*>(codes) + idx, c0);
             }
             if constexpr (DEQ != 0) {
-                const float2 d2s = make_float2(d, d);
+                const float2 d2s = make_float2(d, d), nm2 = make_float2(-kMagic, -kMagic);
                 float2 dq[4];
 #pragma unroll
-                for (int e = 0; e < 4; ++e) dq[e] = __fmul2_rn(q2[e], d2s);
+                for (int e = 0; e < 4; ++e) dq[e] = __fmul2_rn(__fadd2_rn(y2[e], nm2), d2s);
                 if constexpr (DEQ == 1) {
                     uint4 o;
                     o.x = pack16x2<DT>(dq[0].x, dq[0].y); o.y = pack16x2<DT>(dq[1].x, dq[1].y);

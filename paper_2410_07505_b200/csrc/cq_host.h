@@ -14,10 +14,8 @@ struct Plan {
     int nstrips;   // column strips
     int64_t ngroups;  // groups of 4 rows
     int ycap;      // most CTAs per strip the absmax pass may use (rows of the column-partial buffer)
-    size_t off_t, off_c, off_a, off_b, off_ra, off_rb, off_rowpart, off_colpart, off_sync, total;
-    int64_t ymax;  // rows of the column-partial buffer
+    size_t off_t, off_c, off_a, off_b, off_ra, off_rb, off_rowpart, off_colpart, total;
 };
-constexpr size_t kFusedSyncBytes = 256;   // barrier words of the single-launch path for on-chip-sized matrices
 
 Plan make_plan(int64_t T, int64_t I);
 int check_matrix(const void* X, int dtype, int64_t T, int64_t I, int64_t ld);
@@ -36,19 +34,6 @@ struct SmallArgs {
 };
 bool launch_small(const SmallArgs& s, cudaStream_t st);
 int small_stage_fault(unsigned int* fault_host);   // flag of its tile copy
-
-// The single cooperative launch for matrices the chip can hold (cq_fused.cu).  Returns false, having launched
-// nothing, when the shape is not eligible or the driver refuses the launch.  All vector pointers are non-null.
-struct FusedArgs {
-    const void* X; int dtype; int64_t T; int64_t I; int I8; int64_t ld8; int W; int nstrips; int64_t ymax;
-    double alpha; int bits;
-    uint16_t* rowpart; uint16_t* colpart;
-    float *t, *c, *a, *b, *ra, *rb;
-    void* codes; void* deq; int deq_mode; unsigned long long* zero_count;
-    void* sync;
-};
-bool launch_fused(const FusedArgs& f, cudaStream_t st);
-int fused_fault(unsigned int* fault_host);          // flag of its row copies and grid barriers
 
 int scales_from_vectors(int64_t T, int64_t I, const float* t, const float* c, double alpha, int bits,
                         void* workspace, size_t ws_bytes, unsigned long long* to_zero, cudaStream_t st);

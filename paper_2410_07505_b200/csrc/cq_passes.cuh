@@ -14,6 +14,7 @@ namespace cq {
 // `vb` is the block's number; every thread of the CTA calls this with the same vb (it synchronises the CTA).
 constexpr int kK2Cols = 8;       // vector columns per block
 constexpr int kK2Groups = 32;    // partial-row groups per block
+constexpr int kK2Batch = 12;     // partial rows a thread loads at once
 
 template <int DT>
 __device__ __forceinline__ void scales_block(int vb, int64_t T, int64_t I, int I8, int nstrips, int Y, int col_ctas,
@@ -32,11 +33,20 @@ __device__ __forceinline__ void scales_block(int vb, int64_t T, int64_t I, int I
             const int vcol = vb * kK2Cols + vx;
             uint4 m = make_uint4(0, 0, 0, 0);
             if (vcol < I8) {
-#pragma unroll 4
-                for (int y = grp; y < Y; y += kK2Groups) {
-                    const uint4 w = __ldcg(colpart + static_cast<int64_t>(y) * I8 + vcol);
-                    m.x = max_u16x2(m.x, w.x); m.y = max_u16x2(m.y, w.y);
-                    m.z = max_u16x2(m.z, w.z); m.w = max_u16x2(m.w, w.w);
+                // all of a thread's loads (up to kK2Batch per round) are issued before the first is used: the partial
+                // rows come from L2, and a chain of dependent rounds is what this latency-bound step must not have
+                for (int y0 = grp; y0 < Y; y0 += kK2Groups * kK2Batch) {
+                    uint4 w[kK2Batch];
+#pragma unroll
+                    for (int i = 0; i < kK2Batch; ++i) {
+                        const int y = y0 + i * kK2Groups;
+                        w[i] = y < Y ? __ldcg(colpart + static_cast<int64_t>(y) * I8 + vcol) : make_uint4(0, 0, 0, 0);
+                    }
+#pragma unroll
+                    for (int i = 0; i < kK2Batch; ++i) {
+                        m.x = max_u16x2(m.x, w[i].x); m.y = max_u16x2(m.y, w[i].y);
+                        m.z = max_u16x2(m.z, w[i].z); m.w = max_u16x2(m.w, w[i].w);
+                    }
                 }
             }
             s_part[grp][vx] = m;
@@ -104,7 +114,7 @@ __device__ __forceinline__ void quantize_store_row8(const uint4& x, float au, fl
                                                     int64_t vec, void* __restrict__ codes, void* __restrict__ deq,
                                                     unsigned int& zeros) {
     float2 y2[4], q2[4];
-    quantize_row8<DT, BITS, false, LEAN>(x, au, rau, cs.b2, cs.rb2, cs.trusted && rau == rau, y2, q2);
+    quantize_row8<DT, BITS, LEAN>(x, au, rau, cs.b2, cs.rb2, cs.trusted && rau == rau, y2, q2);
     if constexpr (BITS == 8) {
         const uint32_t c0 = pack_int8x4(y2[0].x, y2[0].y, y2[1].x, y2[1].y);
         const uint32_t c1 = pack_int8x4(y2[2].x, y2[2].y, y2[3].x, y2[3].y);

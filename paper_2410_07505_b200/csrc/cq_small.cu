@@ -154,7 +154,7 @@ k_small(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8, int Tc, dou
         const uint4 w = active ? s_x[r * Wv + tid] : make_uint4(0, 0, 0, 0);
         const float au = s_a[r], rau = s_ra[r];
         float2 y2[4], q2[4];
-        quantize_row8<DT, BITS, false, true>(w, au, rau, b2, rb2, cols_trusted && rau == rau, y2, q2);
+        quantize_row8<DT, BITS, true>(w, au, rau, b2, rb2, cols_trusted && rau == rau, y2, q2);
         const int64_t vec = (r0 + r) * I8 + v;
         if constexpr (BITS == 8) {
             const uint32_t c0 = pack_int8x4(y2[0].x, y2[0].y, y2[1].x, y2[1].y);

@@ -71,13 +71,14 @@ k4_weight_rows(const uint4* __restrict__ W, int C8, int64_t ld8,
     const float rd = guarded_rcp(d);
     if (tid == 0 && scale != nullptr) scale[row] = d;
 
-    const float2 ones[4] = {make_float2(1.0f, 1.0f), make_float2(1.0f, 1.0f), make_float2(1.0f, 1.0f), make_float2(1.0f, 1.0f)};
-    const float2 d2s = make_float2(d, d);
+    const float2 d2s = make_float2(d, d), nm2 = make_float2(-kMagic, -kMagic);
+    const bool scale_ok = rd == rd;                   // false: d outside [2^-40, 2^40] (NaN marker)
     unsigned int zeros = 0;
     for (int v = tid; v < C8; v += kThreads) {
         const uint4 w = s_vec[v];
-        float2 y2[4], q2[4];
-        quantize_row8<DT, BITS, true, !BULK>(w, d, rd, ones, ones, rd == rd, y2, q2);
+        float2 y2[4];
+        if (scale_ok) exact_codes_uniform_row8<DT>(w, d, rd, y2);
+        else exact_codes_uniform_slow<DT, BITS>(w, d, y2);                // extreme scale: the whole row, never mixed
         const int64_t vec = row * C8 + v;
         if constexpr (BITS == 8) {
             const uint32_t c0 = pack_int8x4(y2[0].x, y2[0].y, y2[1].x, y2[1].y);
@@ -92,7 +93,7 @@ k4_weight_rows(const uint4* __restrict__ W, int C8, int64_t ld8,
         if constexpr (DEQ != 0) {
             float2 dq[4];
 #pragma unroll
-            for (int k = 0; k < 4; ++k) dq[k] = __fmul2_rn(q2[k], d2s);
+            for (int k = 0; k < 4; ++k) dq[k] = __fmul2_rn(__fadd2_rn(y2[k], nm2), d2s);
             if constexpr (DEQ == 1) {
                 uint4 o;
                 o.x = pack16x2<DT>(dq[0].x, dq[0].y); o.y = pack16x2<DT>(dq[1].x, dq[1].y);

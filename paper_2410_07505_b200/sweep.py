@@ -3,9 +3,12 @@
     python -m paper_2410_07505_b200.sweep                 # every activation config x bit width, 3 weight shapes
     python -m paper_2410_07505_b200.sweep --layers 80     # plus the per-layer sweep (inputs generated per layer)
 
-Times are CUDA-event medians of the public calls with the L2 flushed before every call (a 256 MiB
-write) and also back to back without the flush.  GB/s uses the algorithmic byte counts: activations
-2+2+codes+2 bytes per element (X read twice), weights 2+codes+2 (row read once).  One JSON object per line.
+Times are CUDA-event means of the public calls with the L2 flushed before every call by a 256 MiB read
+(clean lines: the cold number), by a 256 MiB write (126 MB of dirty lines whose write-back competes with
+the call's first pass) and back to back without a flush.  GB/s uses the algorithmic byte counts:
+activations 2+2+codes+2 bytes per element (X read twice; the single-read figure drops one read, for
+matrices L2 can hold), weights 2+codes+2 (row read once).  Every row carries the SM clock sampled while
+it was timed.  One JSON object per line.
 """
 from __future__ import annotations
 
@@ -16,6 +19,7 @@ import statistics
 import numpy as np
 import torch
 
+from . import clocks
 from . import cq
 from . import workloads as wl
 
@@ -26,29 +30,49 @@ def _dev(bits: np.ndarray, dtype: str) -> torch.Tensor:
     return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(TORCH_DT[dtype]).cuda()
 
 
+class L2Flush:
+    """Untimed eviction of L2 between timed calls: `read` leaves clean lines behind, `write` dirty ones."""
+
+    def __init__(self, nbytes: int = 256 << 20, device="cuda"):
+        self.buf = torch.zeros(nbytes, dtype=torch.uint8, device=device)
+        self.words = self.buf.view(torch.int32)
+        self.sum = torch.zeros((), dtype=torch.int64, device=device)
+
+    def read(self) -> None:
+        torch.sum(self.words, dim=0, out=self.sum)
+
+    def write(self) -> None:
+        self.buf.zero_()
+
+
 def _time(fn, flush, iters: int) -> float:
+    """Mean CUDA-event time of `fn` in microseconds; `flush` (a callable or None) runs untimed before every call.
+    (The event clock ticks in steps of about two microseconds here, so a mean resolves what a median cannot.)"""
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
     for _ in range(3):
         fn()
     torch.cuda.synchronize()
     for a, b in ev:
         if flush is not None:
-            flush.zero_()
+            flush()
         a.record()
         fn()
         b.record()
     torch.cuda.synchronize()
-    return statistics.median(a.elapsed_time(b) for a, b in ev) * 1e3     # microseconds
+    return statistics.fmean(a.elapsed_time(b) for a, b in ev) * 1e3     # microseconds
 
 
 def time_activation(Xd: torch.Tensor, bits: int, alpha: float, flush, iters: int) -> dict:
     T, I = Xd.shape
     buf = cq.ActBuffers(T, I, Xd.dtype, bits)
-    us_cold = _time(lambda: cq.quantize_act(Xd, alpha, bits, buffers=buf), flush, iters)
-    us_warm = _time(lambda: cq.quantize_act(Xd, alpha, bits, buffers=buf), None, iters)
+    with clocks.for_current_device() as clk:
+        us_cold = _time(lambda: cq.quantize_act(Xd, alpha, bits, buffers=buf), flush.read, iters)
+        us_dirty = _time(lambda: cq.quantize_act(Xd, alpha, bits, buffers=buf), flush.write, iters)
+        us_warm = _time(lambda: cq.quantize_act(Xd, alpha, bits, buffers=buf), None, iters)
     n = T * I
     per_elem = 2 + 2 + (1 if bits == 8 else 0.5) + 2
-    return {"us_l2_flushed": round(us_cold, 1), "us_back_to_back": round(us_warm, 1),
+    return {"us_l2_flushed": round(us_cold, 1), "us_write_flushed": round(us_dirty, 1), "us_back_to_back": round(us_warm, 1),
+            "sm_mhz": clk.summary()["sm_mhz"],
             "gbs_l2_flushed": round(per_elem * n / us_cold / 1e3, 1),
             "gbs_single_read_accounting": round((per_elem - 2) * n / us_cold / 1e3, 1),
             "elements_per_s": round(n / us_cold * 1e6), "kernel_proportion": int(buf.zero_count.item()) / n}
@@ -56,10 +80,11 @@ def time_activation(Xd: torch.Tensor, bits: int, alpha: float, flush, iters: int
 
 def time_weight(Wd: torch.Tensor, bits: int, flush, iters: int) -> dict:
     out = cq.quantize_weight_per_channel(Wd, bits)
-    us = _time(lambda: cq.quantize_weight_per_channel(Wd, bits, out=out), flush, iters)
+    with clocks.for_current_device() as clk:
+        us = _time(lambda: cq.quantize_weight_per_channel(Wd, bits, out=out), flush.read, iters)
     n = Wd.numel()
     per_elem = 2 + (1 if bits == 8 else 0.5) + 2
-    return {"us_l2_flushed": round(us, 1), "gbs": round(per_elem * n / us / 1e3, 1),
+    return {"us_l2_flushed": round(us, 1), "sm_mhz": clk.summary()["sm_mhz"], "gbs": round(per_elem * n / us / 1e3, 1),
             "kernel_proportion": int(out.zero_count.item()) / n}
 
 
@@ -70,11 +95,11 @@ def time_extra_ops(Xd: torch.Tensor, alpha: float, flush, iters: int) -> dict:
     ws = torch.empty(cq.workspace_bytes(T, I), dtype=torch.uint8, device=Xd.device)
     r = cq.quantize_act(Xd, alpha, 8)
     t, c = cq.absmax_rows_cols(Xd)
-    us_rm = _time(lambda: cq.remove_kernel(Xd, alpha, 8, 1.0, ws), flush, iters)
-    us_ind = _time(lambda: cq.case_indicators(r), flush, iters)
-    us_cnt = _time(lambda: cq.kernel_count_x(Xd, alpha, 8, t, c, ws), flush, iters)
-    us_abs = _time(lambda: cq.absmax_rows_cols(Xd), flush, iters)
-    us_abs_ws = _time(lambda: cq.absmax_rows_cols(Xd, workspace=ws, out=(t, c)), flush, iters)
+    us_rm = _time(lambda: cq.remove_kernel(Xd, alpha, 8, 1.0, ws), flush.read, iters)
+    us_ind = _time(lambda: cq.case_indicators(r), flush.read, iters)
+    us_cnt = _time(lambda: cq.kernel_count_x(Xd, alpha, 8, t, c, ws), flush.read, iters)
+    us_abs = _time(lambda: cq.absmax_rows_cols(Xd), flush.read, iters)
+    us_abs_ws = _time(lambda: cq.absmax_rows_cols(Xd, workspace=ws, out=(t, c)), flush.read, iters)
     _, counts = cq.remove_kernel(Xd, alpha, 8, 1.0, ws)
     ind = cq.case_indicators(r).cpu().tolist()
     cnt = counts.cpu().tolist()
@@ -96,7 +121,7 @@ def time_decode_shapes(flush, iters: int) -> None:
         row = {"shape": [T, I], "dtype": "bf16", "bits": 8}
         for key, no_small in (("one_launch", 0), ("three_launches", 1)):
             cq.set_tuning("no_small", no_small)
-            cold = _time(lambda: cq.quantize_act(Xd, 0.15, 8, buffers=buf), flush, iters)
+            cold = _time(lambda: cq.quantize_act(Xd, 0.15, 8, buffers=buf), flush.read, iters)
             torch.cuda.synchronize()
             t0 = time.perf_counter()
             for _ in range(200):
@@ -125,7 +150,7 @@ def main() -> None:
     ap.add_argument("--decode", action="store_true", help="time decode-sized matrices through the single-launch path, "
                     "the three launches and a CUDA-graph replay, then exit")
     ap.add_argument("--tune", action="append", default=[], metavar="KEY=VALUE",
-                    help="launch-shape knob to set before timing (see cq_set_tuning), e.g. no_fused=1; may be repeated")
+                    help="launch-shape knob to set before timing (see cq_set_tuning), e.g. no_pdl=1; may be repeated")
     ap.add_argument("--only", default="", help="comma-separated config names (e.g. llama70b_mlp,weight_8192x28672): "
                     "time only these (keeps a profiler capture short)")
     args = ap.parse_args()
@@ -134,7 +159,7 @@ def main() -> None:
     for kv in args.tune:
         key, _, value = kv.partition("=")
         cq.set_tuning(key, int(value))
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    flush = L2Flush()
     if args.decode:
         time_decode_shapes(flush, args.iters)
         return
@@ -162,9 +187,10 @@ def main() -> None:
             row.update(time_weight(Wd, bits, flush, args.iters))
             print(json.dumps(row), flush=True)
         out = cq.quantize_weight_groupwise(Wd, 128, 4)
-        us = _time(lambda: cq.quantize_weight_groupwise(Wd, 128, 4, out=out), flush, args.iters)
+        with clocks.for_current_device() as clk:
+            us = _time(lambda: cq.quantize_weight_groupwise(Wd, 128, 4, out=out), flush.read, args.iters)
         print(json.dumps({"config": f"weight_{shape[0]}x{shape[1]}_g128", "shape": list(shape), "dtype": "bf16", "bits": 4,
-                          "us_l2_flushed": round(us, 1), "gbs": round(4.5 * Wd.numel() / us / 1e3, 1),
+                          "us_l2_flushed": round(us, 1), "sm_mhz": clk.summary()["sm_mhz"], "gbs": round(4.5 * Wd.numel() / us / 1e3, 1),
                           "kernel_proportion": int(out.zero_count.item()) / Wd.numel()}), flush=True)
         del Wd, out
 

@@ -8,7 +8,7 @@ with 8 outlier channels x50) are cross-quantized to INT8 and INT4 (alpha = 0.15)
 through the public calls.  Every output of every call (absmax vectors, scale vectors, codes, 16-bit dequantized
 matrix, zero-code count) is compared element by element with the oracle, which sees the same bytes; inputs are
 generated per layer and dropped, so host memory holds one matrix at a time (plus the next one being drawn).
-One JSON object per layer: quantizer time (sum of the 14 calls' CUDA-event medians, L2 flushed before each),
+One JSON object per layer: quantizer time (sum of the 14 calls' mean CUDA-event times, L2 flushed by a 256 MiB read before each),
 the kernel proportions (Definition 1; Section 4.2 averages them over all linear-layer inputs), the number of
 differing elements (must be 0) and the oracle's wall time on the host cores.  This file lives under tests/
 because it runs the oracle; the product package never does.
@@ -67,6 +67,7 @@ def check_layer(layer: int, *, iters: int = 5, time_calls: bool = True, flush=No
     from paper_2410_07505_b200 import cq, sweep, workloads as wl
 
     own_pool = pool is None
+    evict = flush.read if flush is not None else None
     pool = pool or ThreadPoolExecutor(max_workers=1)
     todo = list(_inputs(layer))
     if tokens is not None:
@@ -101,7 +102,7 @@ def check_layer(layer: int, *, iters: int = 5, time_calls: bool = True, flush=No
                          int(zc != ref.zero_count))
                 rec["kernel_proportion_int%d_each" % bits].append(zc / (R * C))
                 if time_calls:
-                    rec["act_us"].append(round(sweep._time(lambda: cq.quantize_act(Md, ALPHA, bits, buffers=buf), flush, iters), 1))
+                    rec["act_us"].append(round(sweep._time(lambda: cq.quantize_act(Md, ALPHA, bits, buffers=buf), evict, iters), 1))
                 del buf, r
             else:
                 out = cq.quantize_weight_per_channel(Md, bits)
@@ -117,7 +118,7 @@ def check_layer(layer: int, *, iters: int = 5, time_calls: bool = True, flush=No
                          int(zc != ref.zero_count))
                 rec["weight_kernel_proportion_int%d_each" % bits].append(zc / (R * C))
                 if time_calls:
-                    rec["weight_us"].append(round(sweep._time(lambda: cq.quantize_weight_per_channel(Md, bits, out=out), flush, iters), 1))
+                    rec["weight_us"].append(round(sweep._time(lambda: cq.quantize_weight_per_channel(Md, bits, out=out), evict, iters), 1))
                 del out
             rec["differences"] += diffs
             rec["elements_compared"] += R * C
@@ -146,7 +147,7 @@ def write_table(path: str, records: list, summary: dict, command: str) -> None:
         "Per layer: 4 activations (2048x8192 x3, 2048x28672; bf16 Laplace, 8 outlier channels x50, alpha = 0.15) x {INT8, INT4}",
         "through `cq_quantize_act` (t, c, scale vectors, codes, bf16 dequantized, count) and 3 weights (8192x8192, 8192x28672,",
         "28672x8192; bf16 N(0, 0.02^2)) x {INT8, INT4} through `cq_quantize_weight_per_channel` (scale, codes, bf16 dequantized,",
-        "count).  Time = sum of the 14 calls' CUDA-event medians, L2 flushed before every call.  Every output element of every",
+        "count).  Time = sum of the 14 calls' mean CUDA-event times, L2 flushed (256 MiB read) before every call.  Every output element of every",
         "call is compared with the CPU oracle on the same bytes; `diff` is the number of differing elements.",
         "",
         f"* layers run: {summary['layers_run']}, elements compared: {summary['elements_compared']:,}, differing: "
@@ -188,7 +189,8 @@ def main() -> int:
     oracle_build.build()
     cuda_build.build()
     cq.lib()
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    from paper_2410_07505_b200 import sweep
+    flush = sweep.L2Flush()
     records = []
     with ThreadPoolExecutor(max_workers=1) as pool, clocks.for_current_device(0.05) as clk:
         for layer in range(0, args.layers, max(1, args.stride)):

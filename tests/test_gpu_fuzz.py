@@ -62,7 +62,6 @@ def test_random_cases_through_every_quantizer(cq, seed):
         T, I = X.shape
         where = (seed, case, dtype, T, I, bits, alpha, theta)
         Xd = to_dev(X, dtype)
-        cq.set_tuning("no_fused", case % 2)                  # alternate between the single launch and the three launches
         r = cq.quantize_act(Xd, alpha, bits)
         parity.check_act(X, dtype, alpha, bits, t=r.t.cpu().numpy(), c=r.c.cpu().numpy(), a=r.row_scale.cpu().numpy(),
                          b=r.col_scale.cpu().numpy(), codes=r.codes.cpu().numpy(), deq=bits_of(r.deq),
@@ -82,5 +81,4 @@ def test_random_cases_through_every_quantizer(cq, seed):
             g = cq.quantize_weight_groupwise(Xd, 128, bits)
             parity.check_weight(X, dtype, bits, scale=g.scale.cpu().numpy(), codes=g.codes.cpu().numpy(),
                                 deq=bits_of(g.deq), zero_count=int(g.zero_count.item()), ref=refg)
-    cq.set_tuning("no_fused", 0)
     assert cq.stage_fault() == 0

@@ -14,15 +14,6 @@ pytestmark = pytest.mark.gpu
 TORCH_DT = {"f16": torch.float16, "bf16": torch.bfloat16}
 
 
-@pytest.fixture(params=["fused", "three_launches"], autouse=True)
-def launch_path(request, cq):
-    """Every test of this file runs twice: matrices the chip can hold take one cooperative launch by default, and
-    the same calls are made with that path switched off (absmax pass, scale vectors, quantize pass)."""
-    cq.set_tuning("no_fused", 1 if request.param == "three_launches" else 0)
-    yield request.param
-    cq.set_tuning("no_fused", 0)
-
-
 def to_dev(bits: np.ndarray, dtype: str) -> torch.Tensor:
     return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(TORCH_DT[dtype]).cuda()
 
