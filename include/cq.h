@@ -12,7 +12,10 @@
  *   - Matrices are row-major, 16-bit (IEEE binary16 or bfloat16), `ld` = distance between rows
  *     in elements (ld >= columns).  Sizes are 64-bit.  Inputs are expected to be finite.
  *   - Every data pointer is a DEVICE pointer owned by the caller.  The library allocates
- *     nothing, frees nothing and keeps no per-call state.
+ *     nothing, frees nothing and keeps no per-call state.  The only state it has is process-wide
+ *     and for measurement: the knobs of cq_set_tuning and the event pair of cq_set_timing_events
+ *     (both thread-safe, neither changes a result), the sticky health flag read by cq_stage_fault,
+ *     and the fixed scratch array of cq_quantize_act_noalloc.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All work is
  *     enqueued on it; no call synchronises; scalar results are written to device memory.
  *   - The return value is a cq_status.  On any status other than CQ_OK no kernel was launched
@@ -240,7 +243,8 @@ int cq_remove_kernel(const void* X, int dtype, int64_t T, int64_t I, int64_t ld,
 int cq_case_indicators(const float* t, const float* c, const float* row_scale, const float* col_scale,
                        int64_t T, int64_t I, int bits, unsigned long long* counts, void* stream);
 
-/* Launch-shape knobs for measurement.  Results never depend on them.  key:
+/* Launch-shape knobs for measurement.  Results never depend on them.  They are PROCESS-WIDE: every later call
+ * of every thread uses them (each call reads a knob once, atomically); leave them alone in production.  key:
  *   "k1_ctas_per_sm", "k3_ctas_per_sm"  resident CTAs per SM the two passes size their grids for (1..64); for the
  *                                       staged quantize pass 2 or 3 picks the build for that occupancy
  *   "k3_forward"  1: the quantize pass walks the rows in ascending order
@@ -256,12 +260,16 @@ int cq_set_tuning(const char* key, int value);
  * (cq_remove_kernel, cq_kernel_count_x) and the weight quantizer on long rows wait for their asynchronous
  * row copies with a bounded number of polls;
  * if a wait ever gives up, a device flag is raised (results of that call are then undefined).  This
- * copies the flag of the current device to *fault_host (0 = never happened).  Synchronises the device. */
+ * copies the flag of the current device to *fault_host (0 = never happened).  Synchronises the device.
+ * A CTA whose wait gave up stops issuing copies, waits once more (bounded) for those in flight and leaves; the
+ * flag is sticky for the life of the process. */
 int cq_stage_fault(unsigned int* fault_host);
 
-/* Measurement hook: while both are non-NULL, cq_quantize_act records the two cudaEvent_t (passed
- * as void*, owned by the caller) on its stream immediately before and after the quantize pass, so
- * that pass can be timed inside a real call.  Pass NULL, NULL to switch it off (the default). */
+/* Measurement hook, PROCESS-WIDE like the knobs above: while both are non-NULL, every cq_quantize_act (of any
+ * thread) records the two cudaEvent_t (passed as void*, owned by the caller) on its stream immediately before and
+ * after the quantize pass, so that pass can be timed inside a real call.  While the hook is set, decode-sized
+ * matrices take the three launches too (the single-launch path has no separate quantize pass to bracket); results
+ * are the same.  Pass NULL, NULL to switch it off (the default).  Setting and reading the pair is thread-safe. */
 int cq_set_timing_events(void* before_quantize_pass, void* after_quantize_pass);
 
 #ifdef __cplusplus

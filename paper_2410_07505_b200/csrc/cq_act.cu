@@ -9,7 +9,9 @@
 // of zero codes.
 #include <math.h>
 
+#include <atomic>
 #include <initializer_list>
+#include <mutex>
 
 #include "cq_common.cuh"
 #include "cq_host.h"
@@ -144,11 +146,12 @@ k1_absmax(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8, int nstri
 // General shapes / alignments: one column per thread, scalar loads, atomic combine (t, c pre-zeroed).
 template <int DT>
 __global__ void __launch_bounds__(kThreads)
-g1_absmax(const uint16_t* __restrict__ X, int64_t T, int64_t I, int64_t ld, int R,
+g1_absmax(const uint16_t* __restrict__ X, int64_t T, int64_t I, int64_t ld, int R, unsigned col_blocks,
           float* __restrict__ t, float* __restrict__ c) {
-    const int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    // one-dimensional grid (row blocks x column blocks fit in 2^31 - 1, not in the 65,535 of the other dimensions)
+    const int64_t j = static_cast<int64_t>(blockIdx.x % col_blocks) * blockDim.x + threadIdx.x;
     const bool active = j < I;
-    const int64_t r0 = static_cast<int64_t>(blockIdx.y) * R;
+    const int64_t r0 = static_cast<int64_t>(blockIdx.x / col_blocks) * R;
     const int64_t r1 = min(T, r0 + R);
     uint32_t cm = 0;
     for (int64_t r = r0; r < r1; ++r) {
@@ -411,13 +414,21 @@ g3_quantize(const uint16_t* __restrict__ X, int64_t T, int64_t I, int64_t ld, in
 }
 
 // ============================================================================ host side
-static int g_tune_k1_ctas = 0;      // resident CTAs per SM assumed for pass 1 (0 = ask the runtime)
-static int g_tune_k3_ctas = 0;      // the same for pass 2
-static int g_tune_k3_forward = 0;   // walk pass 2 in ascending row order
-static int g_tune_no_pdl = 0;       // launch pass 2 without programmatic dependent launch
-static int g_tune_no_small = 0;     // never take the single-launch path for small matrices
-static int g_tune_no_stage = 0;     // pass 2 loads rows straight into registers instead of staging them
-static cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
+// Process-wide measurement settings (cq_set_tuning, cq_set_timing_events).  They never change a result; each is
+// read once per call, atomically, so a call sees one consistent value even if another thread sets it meanwhile.
+static std::atomic<int> g_tune_k1_ctas{0};      // resident CTAs per SM assumed for pass 1 (0 = ask the runtime)
+static std::atomic<int> g_tune_k3_ctas{0};      // the same for pass 2
+static std::atomic<int> g_tune_k3_forward{0};   // walk pass 2 in ascending row order
+static std::atomic<int> g_tune_no_pdl{0};       // launch pass 2 without programmatic dependent launch
+static std::atomic<int> g_tune_no_small{0};     // never take the single-launch path for small matrices
+static std::atomic<int> g_tune_no_stage{0};     // pass 2 loads rows straight into registers instead of staging them
+struct TimingEvents { cudaEvent_t before = nullptr, after = nullptr; };
+static TimingEvents g_events;                   // both or neither, under g_events_mutex
+static std::mutex g_events_mutex;
+static TimingEvents timing_events() {
+    std::lock_guard<std::mutex> lock(g_events_mutex);
+    return g_events;
+}
 
 static inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
@@ -461,6 +472,7 @@ Plan make_plan(int64_t T, int64_t I) {
 }
 
 static bool aligned(const void* p, size_t n) { return (reinterpret_cast<uintptr_t>(p) % n) == 0; }
+constexpr int64_t kMaxGridX = (int64_t(1) << 31) - 1;      // most blocks a one-dimensional grid may have
 
 int check_matrix(const void* X, int dtype, int64_t T, int64_t I, int64_t ld) {
     if (T < 0 || I < 0 || ld < I) return CQ_ERR_SHAPE;
@@ -508,7 +520,7 @@ static int launch_k1(const Plan& p, const void* X, int64_t T, int64_t ld, uint16
                      float* t, float* c, cudaStream_t st) {
     auto kern = k1_absmax<ATOMIC, DT>;
     static thread_local LaunchMemo memo;
-    const int Y = resident_y(kern, p.W, p.nstrips, (p.ngroups * 4 + kG1 - 1) / kG1, g_tune_k1_ctas, ATOMIC ? 0 : p.ycap, memo);
+    const int Y = resident_y(kern, p.W, p.nstrips, (p.ngroups * 4 + kG1 - 1) / kG1, g_tune_k1_ctas.load(), ATOMIC ? 0 : p.ycap, memo);
     kern<<<dim3(p.nstrips, Y), p.W, 0, st>>>(static_cast<const uint4*>(X), T, p.I8, ld / 8, p.nstrips, rowpart,
                                              reinterpret_cast<uint4*>(colpart), t, c);
     return Y;
@@ -526,11 +538,13 @@ static int absmax_atomic(const void* X, int dtype, int64_t T, int64_t I, int64_t
         else launch_k1<true, CQ_BF16>(p, X, T, ld, nullptr, nullptr, t, c, st);
     } else {
         const int R = 64;
-        dim3 grid(static_cast<unsigned>((I + kThreads - 1) / kThreads), static_cast<unsigned>((T + R - 1) / R));
+        const int64_t col_blocks = (I + kThreads - 1) / kThreads, row_blocks = (T + R - 1) / R;
+        if (col_blocks * row_blocks > kMaxGridX) return CQ_ERR_SHAPE;
+        const unsigned grid = static_cast<unsigned>(col_blocks * row_blocks), cb = static_cast<unsigned>(col_blocks);
         if (dtype == CQ_F16)
-            g1_absmax<CQ_F16><<<grid, kThreads, 0, st>>>(static_cast<const uint16_t*>(X), T, I, ld, R, t, c);
+            g1_absmax<CQ_F16><<<grid, kThreads, 0, st>>>(static_cast<const uint16_t*>(X), T, I, ld, R, cb, t, c);
         else
-            g1_absmax<CQ_BF16><<<grid, kThreads, 0, st>>>(static_cast<const uint16_t*>(X), T, I, ld, R, t, c);
+            g1_absmax<CQ_BF16><<<grid, kThreads, 0, st>>>(static_cast<const uint16_t*>(X), T, I, ld, R, cb, t, c);
     }
     return launch_status();
 }
@@ -570,7 +584,7 @@ static bool launch_k3_staged(const Plan& p, const K3Args& k, cudaStream_t st) {
     if (y > 65535) y = 65535;
     if (y < 1) y = 1;
     launch_dependent(kern, dim3(p.nstrips, static_cast<unsigned>(y)), dim3(p.W), smem, st, k.X, k.T, k.I8, k.ld8, k.a, k.ra,
-                     k.b, k.rb, k.codes, k.deq, k.zc, g_tune_k3_forward);
+                     k.b, k.rb, k.codes, k.deq, k.zc, g_tune_k3_forward.load());
     return true;
 }
 
@@ -581,16 +595,17 @@ static void launch_k3_one(const Plan& p, const K3Args& k, cudaStream_t st) {
         // codes the two-CTA build is the faster one at every size measured)
         const int64_t bytes = k.T * k.ld8 * 16;
         int mode = (bytes > (int64_t(120) << 20) || BITS == 4) ? 2 : 3;
-        if (g_tune_k3_ctas == 2 || g_tune_k3_ctas == 3) mode = g_tune_k3_ctas;
+        const int tuned = g_tune_k3_ctas;
+        if (tuned == 2 || tuned == 3) mode = tuned;
         const bool ok = mode == 2 ? launch_k3_staged<DT, BITS, DEQ, CODES, COUNT, 2>(p, k, st)
                                   : launch_k3_staged<DT, BITS, DEQ, CODES, COUNT, 3>(p, k, st);
         if (ok) return;
     }
     auto kern = k3_quantize<DT, BITS, DEQ, CODES, COUNT, 0>;
     static thread_local LaunchMemo memo;
-    const int Y = resident_y(kern, p.W, p.nstrips, p.ngroups, g_tune_k3_ctas, 0, memo);
+    const int Y = resident_y(kern, p.W, p.nstrips, p.ngroups, g_tune_k3_ctas.load(), 0, memo);
     launch_dependent(kern, dim3(p.nstrips, Y), dim3(p.W), 0, st, k.X, k.T, k.I8, k.ld8, k.a, k.ra, k.b, k.rb, k.codes,
-                     k.deq, k.zc, g_tune_k3_forward);
+                     k.deq, k.zc, g_tune_k3_forward.load());
 }
 
 template <int DT, int BITS, int DEQ>
@@ -687,7 +702,9 @@ int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
     const unsigned k2v_blocks = static_cast<unsigned>((T + I + kThreads - 1) / kThreads);
 
     // ---- small matrices: everything in one launch of one thread-block cluster
-    if (!given && fast_in && fast_out && !g_tune_no_small && (g_ev_before == nullptr || g_ev_after == nullptr) &&
+    const TimingEvents ev = timing_events();
+    const bool timed = ev.before != nullptr && ev.after != nullptr;
+    if (!given && fast_in && fast_out && !g_tune_no_small && !timed &&
         (codes != nullptr || deq != nullptr || zero_count != nullptr)) {      // (callers without outputs want the workspace vectors)
         const SmallArgs sa{X, dtype, T, p.I8, ld / 8, p.W, p.nstrips, alpha, bits, t_dev, c_dev, a_dev, b_dev,
                            codes, deq, deq == nullptr ? 0 : (deq_dtype == CQ_F32 ? 2 : 1), zero_count};
@@ -730,8 +747,7 @@ int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
     // ---- pass 2
     const bool any_out = codes != nullptr || deq != nullptr || zero_count != nullptr;
     if (any_out) {
-        const bool timed = g_ev_before != nullptr && g_ev_after != nullptr;
-        if (timed) cudaEventRecord(g_ev_before, st);
+        if (timed) cudaEventRecord(ev.before, st);
         if (fast_in && fast_out) {
             const int deq_mode = deq == nullptr ? 0 : (deq_dtype == CQ_F32 ? 2 : 1);
             const K3Args k{static_cast<const uint4*>(X), T, p.I8, ld / 8, a_dev, ra_dev, b_dev, rb_dev, codes, deq, zero_count};
@@ -744,6 +760,7 @@ int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
             }
         } else {
             const int64_t n = T * ((I + 1) / 2);
+            if ((n + kThreads - 1) / kThreads > kMaxGridX) return CQ_ERR_SHAPE;
             const unsigned blocks = static_cast<unsigned>((n + kThreads - 1) / kThreads);
             if (dtype == CQ_F16)
                 g3_quantize<CQ_F16><<<blocks, kThreads, 0, st>>>(static_cast<const uint16_t*>(X), T, I, ld, bits, a_dev, b_dev,
@@ -752,7 +769,7 @@ int quantize_act_impl(const void* X, int dtype, int64_t T, int64_t I, int64_t ld
                 g3_quantize<CQ_BF16><<<blocks, kThreads, 0, st>>>(static_cast<const uint16_t*>(X), T, I, ld, bits, a_dev, b_dev,
                                                                   codes, deq, deq_dtype, zero_count);
         }
-        if (timed) cudaEventRecord(g_ev_after, st);
+        if (timed) cudaEventRecord(ev.after, st);
         if ((rc = launch_status()) != CQ_OK) return rc;
     }
     if (c != nullptr && !c_in_place && !given) {
@@ -816,8 +833,10 @@ int cq_stage_fault(unsigned int* fault_host) {
 }
 
 int cq_set_timing_events(void* before_quantize_pass, void* after_quantize_pass) {
-    cq::g_ev_before = static_cast<cudaEvent_t>(before_quantize_pass);
-    cq::g_ev_after = static_cast<cudaEvent_t>(after_quantize_pass);
+    std::lock_guard<std::mutex> lock(cq::g_events_mutex);
+    const bool both = before_quantize_pass != nullptr && after_quantize_pass != nullptr;
+    cq::g_events.before = both ? static_cast<cudaEvent_t>(before_quantize_pass) : nullptr;
+    cq::g_events.after = both ? static_cast<cudaEvent_t>(after_quantize_pass) : nullptr;
     return CQ_OK;
 }
 

@@ -3,8 +3,8 @@
     python -m paper_2410_07505_b200.sweep                 # every activation config x bit width, 3 weight shapes
     python -m paper_2410_07505_b200.sweep --layers 80     # plus the per-layer sweep (inputs generated per layer)
 
-Times are CUDA-event means of the public calls with the L2 flushed before every call by a 256 MiB read
-(clean lines: the cold number), by a 256 MiB write (126 MB of dirty lines whose write-back competes with
+Times are CUDA-event means of the public calls with the L2 flushed before every call by reading a 256 MiB buffer
+twice (clean lines: the cold number), by a 256 MiB write (126 MB of dirty lines whose write-back competes with
 the call's first pass) and back to back without a flush.  GB/s uses the algorithmic byte counts:
 activations 2+2+codes+2 bytes per element (X read twice; the single-read figure drops one read, for
 matrices L2 can hold), weights 2+codes+2 (row read once).  Every row carries the SM clock sampled while
@@ -35,11 +35,12 @@ class L2Flush:
 
     def __init__(self, nbytes: int = 256 << 20, device="cuda"):
         self.buf = torch.zeros(nbytes, dtype=torch.uint8, device=device)
-        self.words = self.buf.view(torch.int32)
+        self.words = self.buf.view(torch.int64)      # summed as it is (a narrower type would be widened into a temporary first)
         self.sum = torch.zeros((), dtype=torch.int64, device=device)
 
     def read(self) -> None:
-        torch.sum(self.words, dim=0, out=self.sum)
+        for _ in range(2):        # a single pass over 256 MiB still leaves some of the previous call's dirty lines in L2
+            torch.sum(self.words, dim=0, out=self.sum)
 
     def write(self) -> None:
         self.buf.zero_()

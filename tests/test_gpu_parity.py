@@ -225,6 +225,10 @@ def test_tall_and_wide_extremes(cq):
         X = wl.small_matrix(T, I, "f16", 15, outlier_cols=1)
         run_and_check(cq, X, "f16", 0.15, 8)
         run_and_check(cq, X, "f16", 0.5, 4)
+    # more than 65,535 blocks of 64 rows through the general (unaligned) kernels: their grids are one-dimensional
+    X = wl.small_matrix(4_200_000, 2, "bf16", 16, outlier_cols=1)
+    run_and_check(cq, X, "bf16", 0.15, 8)
+    run_and_check(cq, X, "bf16", 0.5, 4)
 
 
 def test_repeated_calls_reuse_buffers(cq):

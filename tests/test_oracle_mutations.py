@@ -33,6 +33,15 @@ MUTATIONS = {
     "dequant_uses_row_factor_only": ("float xhat = (s == 0.0f) ? 0.0f : (float)q * s;\n            if (q == 0) zeros",
                                      "float xhat = (s == 0.0f) ? 0.0f : (float)q * aa[i];\n            if (q == 0) zeros"),
     "zero_scale_not_guarded": ("if (s == 0.0f) return 0;", ""),
+    "col_abs_dropped": ("float ax = fabsf(decode16(X[i * ld + j], dtype));\n            if (ax > m) m = ax;\n        }\n        c[j] = m;",
+                        "float ax = decode16(X[i * ld + j], dtype);\n            if (ax > m) m = ax;\n        }\n        c[j] = m;"),
+    # Remove Kernel (Figure 1 / Appendix B) and the Table 1 indicators
+    "remove_kernel_bound_is_strict": ("int gone = fabsf(u) <= half_bound;", "int gone = fabsf(u) < half_bound;"),
+    "remove_kernel_bound_not_halved": ("float half_bound = 0.5f * bound_scale;", "float half_bound = bound_scale;"),
+    "remove_kernel_per_token_scale_from_column_maxima": ("float s_pt = t[i] / (float)qmax;\n        for (int64_t j = 0; j < I; ++j) {\n            uint16_t bits16",
+                                                          "float s_pt = c[i % I] / (float)qmax;\n        for (int64_t j = 0; j < I; ++j) {\n            uint16_t bits16"),
+    "case_two_is_strict": ("if (c[j] >= t[i]) n_case2 += 1;", "if (c[j] > t[i]) n_case2 += 1;"),
+    "case_bounds_swapped": ("if (0.5f * s < 0.5f * s_pt) n_smaller += 1;", "if (0.5f * s_pt < 0.5f * s) n_smaller += 1;"),
     # alpha = 0 evaluated through the general branch: s = fl32(fl32(1/qmax) * c) instead of fl32(c/qmax)
     "alpha_zero_not_special_cased": [("else if (alpha == 0.0) a[i] = 1.0f;", ""),
                                      ("else if (alpha == 0.0) b[j] = c[j] / (float)qmax;", "")],

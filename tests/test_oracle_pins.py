@@ -16,6 +16,7 @@ from fractions import Fraction
 import numpy as np
 import pytest
 
+import codecs16
 from oracle import cq_oracle as orc
 from paper_2410_07505_b200 import workloads as wl
 
@@ -23,8 +24,8 @@ QMAX = {8: 127, 4: 7}
 
 
 def dec(bits, dtype):
-    """Decoder that is not the oracle's: numpy (fp16) / bit shift (bf16)."""
-    return wl.bits_to_f32(bits, dtype)
+    """Decoder that is not the oracle's: numpy (fp16) / widened bit pattern (bf16), tests/codecs16.py."""
+    return codecs16.bits_to_f32(bits, dtype)
 
 
 def rand_matrix(T, I, dtype, seed, **kw):
@@ -158,7 +159,7 @@ def test_hand_worked_2x2_example():
       INT8: 127/sqrt(12) = 36.66, 381/sqrt(24) = 77.77, -508/sqrt(32) = -89.80, 1016/sqrt(64) = 127
       INT4:   7/sqrt(12) =  2.02,  21/sqrt(24) =  4.29,  -28/sqrt(32) =  -4.95,   56/sqrt(64) = 7
     none of them near a rounding boundary."""
-    X = wl.to_bits(np.array([[1, 3], [-4, 8]], dtype=np.float32), "f16")
+    X = codecs16.to_bits(np.array([[1, 3], [-4, 8]], dtype=np.float32), "f16")
     r8 = orc.quantize_act(X, "f16", 0.5, 8)
     assert r8.t.tolist() == [3.0, 8.0] and r8.c.tolist() == [4.0, 8.0]
     assert r8.codes.tolist() == [[37, 78], [-90, 127]]
@@ -175,7 +176,7 @@ def test_ties_round_to_even_as_in_the_listing():
     """Appendix B.1's listing rounds with torch.round (ties to even).  With alpha = 1 and a row
     maximum of 127 the step is exactly 1, so u = x and the ties are exact."""
     row = np.array([[127, 0.5, 1.5, 2.5, -0.5, -1.5, -2.5, 3.5, 126.5, -125.5]], dtype=np.float32)
-    r = orc.quantize_act(wl.to_bits(row, "f16"), "f16", 1.0, 8)
+    r = orc.quantize_act(codecs16.to_bits(row, "f16"), "f16", 1.0, 8)
     assert r.codes.tolist() == [[127, 0, 2, 2, 0, -2, -2, 4, 126, -126]]
     assert r.zero_count == 2            # |u| = 1/2 exactly lands in the kernel under this reading
 
@@ -185,7 +186,7 @@ def test_kernel_example_small_values_fall_to_zero_only_per_token():
     cross scale keeps them (the situation of the paper's Section 4.2 discussion)."""
     x = np.full((4, 8), 0.3, dtype=np.float32)
     x[:, 5] = 100.0
-    X = wl.to_bits(x, "f16")
+    X = codecs16.to_bits(x, "f16")
     per_token = orc.quantize_act(X, "f16", 1.0, 8)
     cross = orc.quantize_act(X, "f16", 0.15, 8)
     assert per_token.zero_count == 4 * 7        # 0.3 * 127 / 100 = 0.381 < 1/2
@@ -291,7 +292,7 @@ def test_power_of_two_rescaling_is_exact():
     """t, c, s scale by 2^k exactly when alpha's powers stay exact: alpha = 0.5, k even."""
     X = rand_matrix(16, 16, "bf16", 91, outlier_cols=1)
     x = dec(X, "bf16")
-    X4 = wl.to_bits(x * np.float32(16.0), "bf16")
+    X4 = codecs16.to_bits(x * np.float32(16.0), "bf16")
     r, r4 = orc.quantize_act(X, "bf16", 0.5, 8), orc.quantize_act(X4, "bf16", 0.5, 8)
     assert np.array_equal(r4.t, r.t * 16) and np.array_equal(r4.c, r.c * 16)
     # codes may differ only through the last-bit rounding of pow; they must agree almost everywhere
@@ -328,7 +329,7 @@ def test_alpha_half_against_exact_integer_arithmetic_all_2x2(bits):
     checked = flagged = 0
     for ks in itertools.product(alphabet, repeat=4):
         k = np.array(ks, dtype=np.int64).reshape(2, 2)
-        X = wl.to_bits((k / 4.0).astype(np.float32), "f16")
+        X = codecs16.to_bits((k / 4.0).astype(np.float32), "f16")
         r = orc.quantize_act(X, "f16", 0.5, bits, want_deq32=False, want_deq16=False)
         kt = np.abs(k).max(axis=1)
         kc = np.abs(k).max(axis=0)
@@ -350,7 +351,7 @@ def test_alpha_half_against_exact_integer_arithmetic_random_2x3(bits):
     qmax = QMAX[bits]
     for _ in range(3000):
         k = rng.integers(-12, 13, size=(2, 3))
-        X = wl.to_bits((k / 4.0).astype(np.float32), "bf16")
+        X = codecs16.to_bits((k / 4.0).astype(np.float32), "bf16")
         r = orc.quantize_act(X, "bf16", 0.5, bits, want_deq32=False, want_deq16=False)
         kt, kc = np.abs(k).max(axis=1), np.abs(k).max(axis=0)
         for i in range(2):
@@ -441,13 +442,13 @@ def test_dequantize_reproduces_the_fused_output():
         out32, out16 = orc.dequantize(stored, bits, 30, 44, r.a, r.b, "bf16")
         assert np.array_equal(out32.view(np.uint32), r.deq32.view(np.uint32))
         assert np.array_equal(out16, r.deq16)
-        assert np.array_equal(r.deq16, wl.f32_to_bf16_bits(r.deq32))
+        assert np.array_equal(r.deq16, codecs16.f32_to_bf16_bits(r.deq32))
 
 
 def test_deq16_is_deq32_rounded_once_fp16():
     X = rand_matrix(30, 44, "f16", 502)
     r = orc.quantize_act(X, "f16", 0.15, 8)
-    assert np.array_equal(r.deq16, wl.f32_to_f16_bits(r.deq32))
+    assert np.array_equal(r.deq16, codecs16.f32_to_f16_bits(r.deq32))
 
 
 def test_bad_arguments_are_rejected():
@@ -504,7 +505,7 @@ def test_case_indicators_brute_force_and_relations():
     r1 = orc.quantize_act(X, "bf16", 1.0, 8, want_deq32=False, want_deq16=False)
     assert orc.case_indicators(r1.t, r1.c, r1.a, r1.b, 8)[1] == 0
     # hand example: t = (2, 8), c = (4, 8): pairs with c >= t: (0,0), (0,1), (1,1)
-    Xh = wl.to_bits(np.array([[1, 2], [-4, 8]], dtype=np.float32), "f16")
+    Xh = codecs16.to_bits(np.array([[1, 2], [-4, 8]], dtype=np.float32), "f16")
     rh = orc.quantize_act(Xh, "f16", 0.5, 8)
     assert orc.case_indicators(rh.t, rh.c, rh.a, rh.b, 8) == (3, 1)
 
@@ -526,6 +527,21 @@ def test_remove_kernel_zeroes_exactly_the_kernel_and_touches_nothing_else():
     out, removed, k_pt, _ = orc.remove_kernel(X, "f16", 1.0, 8)
     assert removed == k_pt == int((np.abs(u) <= 0.5).sum())
     assert np.array_equal(out, np.where(np.abs(u) <= 0.5, np.uint16(0), X))
+
+
+def test_remove_kernel_hand_example_with_elements_exactly_on_the_bound():
+    """Per-token scale 1 (row maximum 127): |x / s| is |x| itself, so the bound theta / 2 can be hit exactly.
+    An element ON the bound is removed (for theta = 1 it is the tie that rounds half to even, to code 0)."""
+    row = np.array([[127, 0.5, -0.5, 0.75, 1.5, -1.5, 1.25, 2.0]], dtype=np.float32)
+    X = codecs16.to_bits(row, "f16")
+    out, removed, k_pt, k_cq = orc.remove_kernel(X, "f16", 1.0, 8, 1.0)            # bound 1/2
+    assert (removed, k_pt, k_cq) == (2, 2, 2)
+    assert np.array_equal(codecs16.bits_to_f32(out, "f16"), [[127, 0, 0, 0.75, 1.5, -1.5, 1.25, 2.0]])
+    out, removed, k_pt, k_cq = orc.remove_kernel(X, "f16", 1.0, 8, 3.0)            # bound 3/2: +-1.5 go, 2.0 stays
+    assert (removed, k_pt, k_cq) == (6, 2, 2)
+    assert np.array_equal(codecs16.bits_to_f32(out, "f16"), [[127, 0, 0, 0, 0, 0, 0, 2.0]])
+    out, removed, _, _ = orc.remove_kernel(X, "f16", 1.0, 8, 2.5)                  # bound 5/4: 1.25 is on it
+    assert removed == 4 and np.array_equal(codecs16.bits_to_f32(out, "f16"), [[127, 0, 0, 0, 1.5, -1.5, 0, 2.0]])
 
 
 def test_remove_kernel_bound_scale_sweeps_the_proportion():
