@@ -7,10 +7,15 @@ dequantized matrix, zero-code count) on the LLaMA-70B-MLP-shaped activation matr
 algorithmic bytes per second: 7 bytes per element (two compulsory reads of X, one byte of
 codes, two bytes of dequantized output) divided by the device time of the step.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--mode replicas|row_sharded]
 
-With N > 1 (launched by torchrun, one rank per GPU) every rank quantizes its own matrix of the
-same shape: the path has no exchange step, so the ranks are independent (weak scaling).
+With N > 1 there is one rank per GPU: started by torchrun (RANK / LOCAL_RANK / WORLD_SIZE in the
+environment) or, when the script is run directly, by the script itself, which re-launches itself under
+torch.distributed.run on 127.0.0.1.  A world size that does not match --gpus, or fewer GPUs than ranks, is
+an error, never a silent single-GPU run.  Default mode: every rank quantizes its own matrix of the same
+shape -- the path has no exchange step, so the ranks are independent (weak scaling).  --mode row_sharded
+measures the sharded variant instead: ONE matrix of the same shape with its tokens split over the ranks,
+the column maxima combined by an all-reduce MAX between the passes (strong scaling).
 `--impl reference` times the CPU oracle, as it stands, on a bounded sample of the same workload.
 """
 from __future__ import annotations
@@ -121,6 +126,128 @@ def run_reference(args) -> None:
     }))
 
 
+def run_row_sharded(args) -> None:
+    """The sharded variant of the path (tokens of ONE matrix split over the ranks): per step every rank runs the
+    absmax pass on its row block, the column maxima are combined by an all-reduce MAX (I floats, NCCL, into local
+    memory), and every rank quantizes its block with its own t and the combined c; the kernel sizes are summed.
+    Strong scaling: the matrix is the headline one whatever the number of ranks."""
+    import torch
+    import torch.distributed as dist
+
+    from paper_2410_07505_b200 import build as cuda_build, clocks as clk, cq, sharded, workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if local == 0:
+        cuda_build.build()
+    if world > 1:
+        dist.barrier()
+    cq.lib()
+    cfg = rank_config(0)                                   # the same matrix on every rank: each keeps its rows
+    X = wl.generate_activation(cfg)
+    T, I = X.shape
+    r0, r1 = sharded.shard_rows(T, world, rank)
+    Xd = torch.from_numpy(np.ascontiguousarray(X[r0:r1]).view(np.int16)).view(torch.bfloat16).cuda()
+    del X
+    buf = cq.ActBuffers(r1 - r0, I, torch.bfloat16, BITS)
+    flush_words = torch.zeros(L2_FLUSH_BYTES // 8, dtype=torch.int64, device="cuda")
+    flush_sum = torch.zeros((), dtype=torch.int64, device="cuda")
+
+    def step():
+        return sharded.quantize_act_row_sharded(Xd, ALPHA, BITS, buffers=buf)
+
+    def flush_l2():
+        for _ in range(2):
+            torch.sum(flush_words, dim=0, out=flush_sum)
+
+    for _ in range(args.warmup):
+        flush_l2()
+        step()
+    torch.cuda.synchronize()
+    K = args.steps
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    with clk.ClockSampler(local, str(torch.cuda.get_device_properties(local).uuid), period_s=0.002) as clocks:
+        for a_, b_ in ev:
+            flush_l2()
+            a_.record()
+            _, total = step()
+            b_.record()
+        torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    total_ms = max_over_ranks(sum(a_.elapsed_time(b_) for a_, b_ in ev), "cuda")
+    n = T * I
+    value = BYTES_PER_ELEMENT_STEP * n * K / (total_ms * 1e-3) / 1e9          # the whole matrix per step, all ranks together
+    if rank == 0:
+        peak, peak_kind = measured_peak()
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
+            "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic", "mode": "row_sharded",
+            "config": {"workload": workload_name(cfg) + f", tokens split over {world} rank(s)",
+                       "exchange": "all-reduce MAX of the column maxima (I floats) between the passes, all-reduce SUM of the "
+                                   "kernel sizes; NCCL into local memory, no peer-memory operands",
+                       "l2": "flushed between steps by reading a 256 MiB buffer twice, untimed",
+                       "timing": "CUDA events per step on the launch stream, summed; max over ranks"},
+            "fraction_of_hbm_roofline": value / (peak * world), "peak_kind": f"of {peak_kind}",
+            "kernel_proportion": int(total.item()) / n, "clocks": clocks.summary(),
+            "gpu_launches": 3 * K, "e2e": None}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def ensure_ranks(args, argv) -> None:
+    """Make --gpus N mean N ranks.  Under a launcher (WORLD_SIZE set) the world size must equal N; run directly with
+    N > 1, the script starts its own ranks: it replaces itself by torch.distributed.run (one node, rendezvous on
+    127.0.0.1) running the same command line.  Never falls back to fewer ranks."""
+    world = os.environ.get("WORLD_SIZE")
+    if world is not None:
+        if int(world) != args.gpus:
+            sys.exit(f"bench.py: --gpus {args.gpus} but WORLD_SIZE={world}: refusing to run with another number of ranks")
+        return
+    if args.gpus == 1:
+        return
+    if args.gpus < 1:
+        sys.exit("bench.py: --gpus must be at least 1")
+    if not args.dry_run:
+        import torch
+        have = torch.cuda.device_count()
+        if have < args.gpus:
+            sys.exit(f"bench.py: --gpus {args.gpus} but only {have} CUDA device(s) are visible: refusing to run on fewer")
+    os.environ.setdefault("NCCL_DEBUG", "INFO")         # the communicator log (transport, NVLS) goes to stderr with the run
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--standalone", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--local-addr", "127.0.0.1", os.path.abspath(__file__), *argv]
+    sys.stdout.flush()
+    os.execv(sys.executable, cmd)
+
+
+def run_dry(args) -> None:
+    """The rank plumbing alone, on the CPU (gloo): rendezvous, barrier, max over ranks, one JSON line from rank 0."""
+    import torch
+    import torch.distributed as dist
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+        dist.barrier()
+    seen = torch.zeros(world, dtype=torch.int64)
+    seen[rank] = 1
+    if world > 1:
+        dist.all_reduce(seen)
+    slowest = max_over_ranks(1.0 + rank, "cpu")
+    if rank == 0:
+        print(json.dumps({"dry_run": True, "n_gpus": world, "ranks_seen": int(seen.sum()), "max_ms": slowest,
+                          "mode": args.mode, "seeds": [rank_config(r).seed for r in range(world)]}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -128,10 +255,21 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--mode", default="replicas", choices=["replicas", "row_sharded"],
+                    help="replicas: one matrix per rank, no exchange (weak scaling, the headline); row_sharded: one matrix "
+                         "with its tokens split over the ranks and an all-reduce MAX of the column maxima (strong scaling)")
+    ap.add_argument("--dry-run", action="store_true", help="start the ranks, run the rank plumbing on the CPU (gloo) and exit")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+        return
+    ensure_ranks(args, sys.argv[1:])
+    if args.dry_run:
+        run_dry(args)
+        return
+    if args.mode == "row_sharded":
+        run_row_sharded(args)
         return
 
     import torch

@@ -110,3 +110,23 @@ def test_shard_rows_partition():
             assert all(a[1] == b[0] for a, b in zip(spans, spans[1:]))
             sizes = [b - a for a, b in spans]
             assert max(sizes) - min(sizes) <= 1
+
+
+# ---- bench.py --gpus N run directly starts its own N ranks (checked on the CPU through --dry-run) ----
+def test_bench_starts_its_own_ranks_and_never_runs_with_fewer():
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--dry-run"], env=env,
+                       capture_output=True, text=True, cwd=ROOT, timeout=600)
+    assert p.returncode == 0, p.stderr[-3000:]
+    line = json.loads([ln for ln in p.stdout.strip().splitlines() if ln.startswith("{")][-1])
+    assert line["dry_run"] and line["n_gpus"] == 2 and line["ranks_seen"] == 2
+    assert line["max_ms"] == 2.0 and len(set(line["seeds"])) == 2
+    # a launcher's world size that disagrees with --gpus is an error, not a quiet single-rank run
+    env_bad = dict(env, RANK="0", LOCAL_RANK="0", WORLD_SIZE="1")
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--dry-run"], env=env_bad,
+                       capture_output=True, text=True, cwd=ROOT, timeout=120)
+    assert p.returncode != 0 and "WORLD_SIZE" in p.stderr
+    # more ranks than visible GPUs (none here) is refused before anything is started
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "1"], env=dict(env, CUDA_VISIBLE_DEVICES=""),
+                       capture_output=True, text=True, cwd=ROOT, timeout=120)
+    assert p.returncode != 0 and "refusing" in p.stderr
