@@ -118,7 +118,9 @@ k9_zero_tests(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
         auto do_row = [&](const uint4& slot, const float (&thr)[6], int64_t row, int vec) {
             const uint32_t words[4] = {slot.x, slot.y, slot.z, slot.w};
             uint32_t m_c = 0, m_p = 0, m_g = 0;
-            bool undecided = !cols_trusted;
+            // smallest distance of any element from each bound: one three-way minimum per pair and one comparison per
+            // row instead of a comparison per element
+            float near_c = INFINITY, near_p = INFINITY, near_g = INFINITY;
             uint32_t ow[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
@@ -127,26 +129,27 @@ k9_zero_tests(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
                 const float2 p = __fmul2_rn(x, rb2[k]);
                 const float px = fabsf(p.x), py = fabsf(p.y);
                 const float d0 = __fadd_rn(px, -thr[0]), d1 = __fadd_rn(py, -thr[0]);
-                undecided |= fabsf(d0) < thr[1];
-                undecided |= fabsf(d1) < thr[1];
+                near_c = fminf(near_c, fminf(fabsf(d0), fabsf(d1)));
                 uint32_t gone = negative_halves(d0, d1);
                 m_c |= gone & bit;
                 if constexpr (!SAME) {
                     const float g0 = __fadd_rn(px, -thr[4]), g1 = __fadd_rn(py, -thr[4]);
-                    undecided |= fabsf(g0) < thr[5];
-                    undecided |= fabsf(g1) < thr[5];
+                    near_g = fminf(near_g, fminf(fabsf(g0), fabsf(g1)));
                     gone = negative_halves(g0, g1);
                     m_g |= gone & bit;
                 }
                 if constexpr (DUAL) {
                     const float e0 = __fadd_rn(fabsf(x.x), -thr[2]), e1 = __fadd_rn(fabsf(x.y), -thr[2]);
-                    undecided |= fabsf(e0) < thr[3];
-                    undecided |= fabsf(e1) < thr[3];
+                    near_p = fminf(near_p, fminf(fabsf(e0), fabsf(e1)));
                     m_p |= negative_halves(e0, e1) & bit;
                 }
                 ow[k] = words[k] & ~gone;
             }
             unsigned int r_cq = __popc(m_c), r_pt = __popc(m_p), r_rm = SAME ? r_cq : __popc(m_g);
+            // (a NaN distance -- infinite threshold, band of zero -- compares false, exactly as the per-element test did)
+            bool undecided = !cols_trusted || near_c < thr[1];
+            if constexpr (!SAME) undecided |= near_g < thr[5];
+            if constexpr (DUAL) undecided |= near_p < thr[3];
             if (undecided) {
                 // Rare: some element sits within 2^-16 (relative) of a bound, or a scale factor is extreme.
                 // The whole vector is decided again from the IEEE quotients.
