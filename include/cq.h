@@ -147,7 +147,10 @@ int cq_quantize_act_given(const void* X, int dtype, int64_t T, int64_t I, int64_
  *     enqueue nothing.  (4096 x 28672 needs 4.5 MiB; every benchmark configuration fits.)
  *   - First call on a device: it looks up the array's address on the current device (one
  *     cudaGetSymbolAddress, remembered afterwards).  Make that first call with the right device current
- *     and before starting any stream capture.
+ *     and before starting any stream capture.  Make it EARLY, too: the CUDA runtime may load the library's
+ *     device code, and with it these 8 MiB, onto a GPU only when it is first needed there, so a process that
+ *     has already handed the rest of the device's memory to its pool could see CQ_ERR_CUDA from the first
+ *     call.  After that first call nothing more is ever taken (free device memory stays where it was).
  *   - All calls on a device share the one array and find the previous call's contents in it; nothing in
  *     it needs clearing between calls.  Two calls whose kernels may overlap on the GPU (different
  *     streams without an ordering between them) race on the array and give undefined results: keep

@@ -5,8 +5,9 @@
 // a serving process that handed the whole GPU to one pool at start-up, a plug-in running on a hot path
 // where the host framework forbids cudaMalloc (it synchronises the device and can fail when memory is
 // fragmented), a component whose memory budget was fixed before it was loaded.  For them this file
-// keeps the scratch inside the library image: one fixed array per GPU, present from the moment the
-// library is loaded on that GPU until the process exits.
+// keeps the scratch inside the library image: one fixed array per GPU, held from the moment the CUDA
+// runtime has loaded this file's device code on that GPU (at the latest during the first call there,
+// which should therefore come early) until the process exits.
 #include <cuda_runtime.h>
 
 #include <mutex>
