@@ -147,7 +147,7 @@ def write_table(path: str, records: list, summary: dict, command: str) -> None:
         "Per layer: 4 activations (2048x8192 x3, 2048x28672; bf16 Laplace, 8 outlier channels x50, alpha = 0.15) x {INT8, INT4}",
         "through `cq_quantize_act` (t, c, scale vectors, codes, bf16 dequantized, count) and 3 weights (8192x8192, 8192x28672,",
         "28672x8192; bf16 N(0, 0.02^2)) x {INT8, INT4} through `cq_quantize_weight_per_channel` (scale, codes, bf16 dequantized,",
-        "count).  Time = sum of the 14 calls' mean CUDA-event times, L2 flushed (256 MiB read) before every call.  Every output element of every",
+        "count).  Time = sum of the 14 calls' mean CUDA-event times, L2 flushed (a 256 MiB buffer read twice) before every call.  Every output element of every",
         "call is compared with the CPU oracle on the same bytes; `diff` is the number of differing elements.",
         "",
         f"* layers run: {summary['layers_run']}, elements compared: {summary['elements_compared']:,}, differing: "
