@@ -112,6 +112,35 @@ def time_extra_ops(Xd: torch.Tensor, alpha: float, flush, iters: int) -> dict:
             "share_c_ge_t": ind[0] / n, "share_bound_smaller": ind[1] / n}
 
 
+def time_whole_layer(layer: int, alpha: float, iters: int) -> dict:
+    """One layer of the 80-layer sweep the way a pipeline would run it: the seven inputs resident on the device, the 14
+    quantizer calls (4 activations and 3 weights, INT8 and INT4 each) issued back to back on one stream between ONE pair
+    of events -- no flush, no per-call event latency -- and the same 14 calls replayed from one CUDA graph."""
+    acts = [_dev(wl.generate_activation(wl.sweep_activation_config(layer, k)), "bf16") for k in range(4)]
+    weights = [_dev(wl.sweep_weight(layer, k), "bf16") for k in range(3)]
+    abuf = {(k, bits): cq.ActBuffers(X.shape[0], X.shape[1], X.dtype, bits) for k, X in enumerate(acts) for bits in (8, 4)}
+    wout = {(k, bits): cq.quantize_weight_per_channel(W, bits) for k, W in enumerate(weights) for bits in (8, 4)}
+
+    def layer_calls():
+        for k, X in enumerate(acts):
+            for bits in (8, 4):
+                cq.quantize_act(X, alpha, bits, buffers=abuf[(k, bits)])
+        for k, W in enumerate(weights):
+            for bits in (8, 4):
+                cq.quantize_weight_per_channel(W, bits, out=wout[(k, bits)])
+
+    with clocks.for_current_device() as clk:
+        us_calls = _time(layer_calls, None, iters)
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            layer_calls()
+        us_graph = _time(graph.replay, None, iters)
+    elements = sum(X.numel() for X in acts) + sum(W.numel() for W in weights)
+    return {"layer": layer, "whole_layer_back_to_back_us": round(us_calls, 1), "whole_layer_graph_replay_us": round(us_graph, 1),
+            "calls": 14, "elements_per_bit_width": elements, "sm_mhz": clk.summary()["sm_mhz"]}
+
+
 def time_decode_shapes(flush, iters: int) -> None:
     """Decode-sized matrices: CUDA-event time of one call after an L2 flush, wall time per call of 200 calls issued
     back to back (host included), for the single-launch path and the three launches, and per replay of a graph."""
@@ -148,6 +177,8 @@ def main() -> None:
     ap.add_argument("--iters", type=int, default=30)
     ap.add_argument("--layers", type=int, default=0, help="layers of the 80-layer sweep to run (0 = skip)")
     ap.add_argument("--alpha", type=float, default=0.15)
+    ap.add_argument("--whole-layer", action="store_true", help="with --layers: also time each layer's 14 calls issued back to back "
+                    "between ONE pair of events (all seven inputs resident, no flush), and replayed from a CUDA graph")
     ap.add_argument("--decode", action="store_true", help="time decode-sized matrices through the single-launch path, "
                     "the three launches and a CUDA-graph replay, then exit")
     ap.add_argument("--tune", action="append", default=[], metavar="KEY=VALUE",
@@ -197,6 +228,8 @@ def main() -> None:
 
     total_us = 0.0
     for layer in range(args.layers):
+        if args.whole_layer:
+            print(json.dumps(time_whole_layer(layer, args.alpha, max(5, args.iters // 3))), flush=True)
         props = []
         layer_us = 0.0
         for k in range(4):
