@@ -7,6 +7,7 @@
 // rows in the opposite order; the rows arrive through a shared-memory ring filled by asynchronous bulk
 // copies), forms s_ij = a_i * b_j in registers and emits codes, the dequantized matrix and the number
 // of zero codes.
+#include <cooperative_groups.h>
 #include <math.h>
 
 #include <atomic>
@@ -122,6 +123,28 @@ k1_absmax(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8, int nstri
     }
     if (lg > 0) flush_rows(chunk_g0, lg);
 
+    if constexpr (ATOMIC) {
+        // The CTAs of a thread-block cluster (up to 8 along y: the same columns, different rows) first combine their
+        // column maxima through distributed shared memory; only the cluster's first CTA goes to memory, which cuts the
+        // atomics on every column by the cluster size (they were what this variant spent most of its time on).
+        namespace cg = cooperative_groups;
+        cg::cluster_group cluster = cg::this_cluster();
+        const unsigned members = cluster.num_blocks();
+        if (members > 1) {
+            __shared__ uint4 s_cm[kThreads];
+            s_cm[tid] = cm;
+            cluster.sync();
+            if (cluster.block_rank() == 0) {
+                for (unsigned r = 1; r < members; ++r) {
+                    const uint4 o = cluster.map_shared_rank(s_cm, r)[tid];
+                    cm.x = max_u16x2(cm.x, o.x); cm.y = max_u16x2(cm.y, o.y);
+                    cm.z = max_u16x2(cm.z, o.z); cm.w = max_u16x2(cm.w, o.w);
+                }
+            }
+            cluster.sync();                              // nobody's shared memory goes away while it is being read
+            if (cluster.block_rank() != 0) return;
+        }
+    }
     if (active) {
         if constexpr (ATOMIC) {
             if (c != nullptr) {
@@ -140,6 +163,18 @@ k1_absmax(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8, int nstri
         } else {
             colpart[static_cast<int64_t>(blockIdx.y) * I8 + v] = cm;
         }
+    }
+}
+
+// Zeroes the two absmax vectors (the identity of the atomic maxima) in one launch.  Either pointer may be null.
+// (Letting the absmax kernel overlap it as a programmatic dependent gained 1.5 us on 16-42 MB matrices and lost 7 us
+// on 235 MB, so the two are ordinary, ordered launches.)
+__global__ void __launch_bounds__(kThreads)
+k0_zero_vectors(float* __restrict__ t, int64_t T, float* __restrict__ c, int64_t I) {
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+    for (int64_t k = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; k < T + I; k += stride) {
+        if (k < T) { if (t != nullptr) t[k] = 0.0f; }
+        else if (c != nullptr) c[k - T] = 0.0f;
     }
 }
 
@@ -520,7 +555,30 @@ static int launch_k1(const Plan& p, const void* X, int64_t T, int64_t ld, uint16
                      float* t, float* c, cudaStream_t st) {
     auto kern = k1_absmax<ATOMIC, DT>;
     static thread_local LaunchMemo memo;
-    const int Y = resident_y(kern, p.W, p.nstrips, (p.ngroups * 4 + kG1 - 1) / kG1, g_tune_k1_ctas.load(), ATOMIC ? 0 : p.ycap, memo);
+    int Y = resident_y(kern, p.W, p.nstrips, (p.ngroups * 4 + kG1 - 1) / kG1, g_tune_k1_ctas.load(), ATOMIC ? 0 : p.ycap, memo);
+    if constexpr (ATOMIC) {
+        // clusters of up to 8 CTAs along y (a portable size); the grid's y extent becomes a multiple of the cluster's
+        int cy = 8;
+        while (cy > 1 && Y < cy) cy >>= 1;
+        Y = Y / cy * cy;
+        if (cy > 1) {
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = 1;
+            attr[0].val.clusterDim.y = static_cast<unsigned>(cy);
+            attr[0].val.clusterDim.z = 1;
+            cudaLaunchConfig_t cfg{};
+            cfg.gridDim = dim3(p.nstrips, Y);
+            cfg.blockDim = dim3(p.W);
+            cfg.stream = st;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            if (cudaLaunchKernelEx(&cfg, kern, static_cast<const uint4*>(X), T, p.I8, ld / 8, p.nstrips, rowpart,
+                                   reinterpret_cast<uint4*>(colpart), t, c) == cudaSuccess)
+                return Y;
+            cudaGetLastError();                          // refused as a cluster launch: an ordinary one does the same work
+        }
+    }
     kern<<<dim3(p.nstrips, Y), p.W, 0, st>>>(static_cast<const uint4*>(X), T, p.I8, ld / 8, p.nstrips, rowpart,
                                              reinterpret_cast<uint4*>(colpart), t, c);
     return Y;
@@ -529,9 +587,15 @@ static int launch_k1(const Plan& p, const void* X, int64_t T, int64_t ld, uint16
 // pass 1 with atomics into pre-zeroed t / c (either may be null)
 static int absmax_atomic(const void* X, int dtype, int64_t T, int64_t I, int64_t ld, float* t, float* c,
                          cudaStream_t st) {
-    if (t != nullptr && cudaMemsetAsync(t, 0, sizeof(float) * T, st) != cudaSuccess) return CQ_ERR_CUDA;
-    if (c != nullptr && cudaMemsetAsync(c, 0, sizeof(float) * I, st) != cudaSuccess) return CQ_ERR_CUDA;
-    if (T == 0 || I == 0) return CQ_OK;
+    {
+        const int64_t n = (t != nullptr ? T : 0) + (c != nullptr ? I : 0);
+        if (n > 0) {
+            int64_t blocks = (T + I + kThreads - 1) / kThreads;
+            if (blocks > 2 * sm_count()) blocks = 2 * sm_count();
+            k0_zero_vectors<<<static_cast<unsigned>(blocks), kThreads, 0, st>>>(t, T, c, I);
+        }
+    }
+    if (T == 0 || I == 0) return launch_status();
     Plan p = make_plan(T, I);
     if (fast_input(X, I, ld)) {
         if (dtype == CQ_F16) launch_k1<true, CQ_F16>(p, X, T, ld, nullptr, nullptr, t, c, st);
