@@ -12,19 +12,28 @@
 
 namespace cq {
 
-// |fl32(x / s_ij)| <= h, decided without a division where that is safe.  With a_i, b_j in [2^-40, 2^40],
+// Membership in the quantization kernel itself (h = 1/2) needs no division and no tolerance: for a 16-bit element x
+// and a normal fp32 scale s,
+//     |fl32(x / s)| <= 1/2   <=>   |x| <= s / 2.
+// (<=: the quotient of x <= s/2 is at most 1/2 and rounding is monotone.  =>: x and s/2 are both fp32 numbers, so
+// x > s/2 means x >= s/2 + ulp(s/2), i.e. x/s >= 1/2 + ulp(s/2)/s > 1/2 + 2^-25, which rounds to a float above 1/2;
+// the tie 1/2 + 2^-25 itself would need x - s/2 = s 2^-25 < ulp(s/2), which no pair of floats has.)  And since |x| is
+// a 16-bit float, |x| <= s/2 is an integer comparison of its 15-bit pattern with the largest 16-bit float not above
+// s/2 (the fp32 value rounded toward zero to 16 bits).  So the CrossQuant kernel (s_ij = fl32(a_i b_j), its half formed
+// exactly as fl32((a_i / 2) b_j)) and the per-token kernel (one threshold pattern per row from fl32(t_i / qmax) / 2) are
+// decided on the packed 16-bit words: no unpacking, no band, nothing undecided.  Rows or columns whose scale factors
+// lie outside [2^-40, 2^40] (where s / 2 might not be exact) are marked and take the IEEE quotients.
+//
+// A bound other than 1/2 (bound_scale != 1) has no such identity.  There, with a_i, b_j in [2^-40, 2^40],
 // p = fl32(x * (1/b_j)) against the row's threshold m_i = fl32(h a_i) compares like |z| = |x / s_ij| against h
 // up to a relative error of 4 * 2^-24 (the roundings of 1/b_j, p, m_i and s_ij = fl32(a_i b_j)), and fl32(z)
 // lies within 2^-24 |z| of z; so for h in [2^-20, 2^20] (nothing near h can be subnormal) and
 // e_i = fl32(2^-18 h a_i), six times that error,
 //     |p| - m_i <= -e_i  =>  |fl32(z)| < h,        |p| - m_i >= e_i  =>  |fl32(z)| > h,
-// and only elements with | |p| - m_i | < e_i need the quotient itself.  Per-token quantization (one scale
-// per row, fl32(t_i / qmax)) compares |x| with fl32(t_i fl32(h / qmax)) in the same way (one more rounding).
-// A zero scale gives (m, e) = (inf, 0): everything in the row is in the kernel; a scale outside
-// [2^-40, 2^40], or h outside [2^-20, 2^20], gives (0, inf): every element takes the quotient.
-// f[]: what the row's scale (a_i, or t_i for per-token) is multiplied with to get m and e, in the order
-// CrossQuant with h = 1/2, per-token with h = 1/2, CrossQuant with the caller's bound.
-struct ZeroFactors { float f[6]; float inv_qmax; };
+// and only elements with | |p| - m_i | < e_i need the quotient itself.  A zero scale gives (m, e) = (inf, 0):
+// everything in the row is removed; a scale outside [2^-40, 2^40], or h outside [2^-20, 2^20], gives (0, inf): every
+// element takes the quotient.  ZeroFactors: what a_i is multiplied with to get m_i and e_i.
+struct ZeroFactors { float m, e; };
 
 static __device__ __noinline__ bool exact_at_most(float x, float s, float h) {
     if (s == 0.0f) return true;                       // the code of a zero scale is 0 by definition
@@ -39,6 +48,27 @@ __device__ unsigned int g_diag_stage_fault = 0;    // set if a bounded wait on a
 __device__ __forceinline__ uint32_t negative_halves(float d_lo, float d_hi) {
     uint32_t r;
     asm("prmt.b32 %0, %1, %2, 0xFFBB;" : "=r"(r) : "r"(__float_as_uint(d_lo)), "r"(__float_as_uint(d_hi)));
+    return r;
+}
+
+// The largest 16-bit values (fp16 or bf16 patterns) not above two non-negative floats, packed low | high << 16:
+// conversion with rounding toward zero (it saturates at the largest finite fp16); for bf16 that is the upper half
+// of the binary32 pattern.
+template <int DT>
+__device__ __forceinline__ uint32_t floor16x2(float lo, float hi) {
+    if constexpr (DT == CQ_BF16) {
+        return __byte_perm(__float_as_uint(lo), __float_as_uint(hi), 0x7632);
+    } else {
+        uint32_t r;
+        asm("cvt.rz.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+        return r;
+    }
+}
+
+// 0xFFFF in each half of the result whose bit 15 is set in w, else 0 (byte permute replicating the sign of bytes 1 and 3).
+__device__ __forceinline__ uint32_t sign_halves(uint32_t w) {
+    uint32_t r;
+    asm("prmt.b32 %0, %1, %1, 0xBB99;" : "=r"(r) : "r"(w));
     return r;
 }
 
@@ -114,42 +144,53 @@ k9_zero_tests(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
                                   ((rb2[2].x + rb2[2].y) + (rb2[3].x + rb2[3].y)) < INFINITY;
         const uint4* xp = X + vv;
 
-        // thr[]: (m, e) of CrossQuant for 1/2, of per-token quantization, of CrossQuant for half_bound
-        auto do_row = [&](const uint4& slot, const float (&thr)[6], int64_t row, int vec) {
+        // column scale factors of this thread's eight columns
+        float2 b2[4];
+        {
+            const float4* bp = reinterpret_cast<const float4*>(b) + static_cast<int64_t>(vv) * 2;
+            const float4 b0 = __ldg(bp), b1 = __ldg(bp + 1);
+            b2[0] = make_float2(b0.x, b0.y); b2[1] = make_float2(b0.z, b0.w);
+            b2[2] = make_float2(b1.x, b1.y); b2[3] = make_float2(b1.z, b1.w);
+        }
+
+        // thr[]: a_i / 2 (NaN: a_i outside the range), per-token threshold pattern in both halves (all ones: outside
+        // the range), (m, e) of CrossQuant for the caller's bound
+        auto do_row = [&](const uint4& slot, const float (&thr)[4], int64_t row, int vec) {
             const uint32_t words[4] = {slot.x, slot.y, slot.z, slot.w};
+            const float2 ah2 = make_float2(thr[0], thr[0]);
+            const uint32_t tpt2 = __float_as_uint(thr[1]);
             uint32_t m_c = 0, m_p = 0, m_g = 0;
-            // smallest distance of any element from each bound: one three-way minimum per pair and one comparison per
-            // row instead of a comparison per element
-            float near_c = INFINITY, near_p = INFINITY, near_g = INFINITY;
+            float near_g = INFINITY;          // smallest distance of any element from the caller's bound (band test, once per row)
             uint32_t ow[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                const uint32_t bit = 0x00010001u << k;
-                const float2 x = unpack16x2<DT>(words[k]);
-                const float2 p = __fmul2_rn(x, rb2[k]);
-                const float px = fabsf(p.x), py = fabsf(p.y);
-                const float d0 = __fadd_rn(px, -thr[0]), d1 = __fadd_rn(py, -thr[0]);
-                near_c = fminf(near_c, fminf(fabsf(d0), fabsf(d1)));
-                uint32_t gone = negative_halves(d0, d1);
-                m_c |= gone & bit;
-                if constexpr (!SAME) {
-                    const float g0 = __fadd_rn(px, -thr[4]), g1 = __fadd_rn(py, -thr[4]);
+                // |x| as a 15-bit pattern against the largest 16-bit value <= s / 2: bit 15 of each half of
+                // (threshold + 0x8000 - magnitude) is set exactly where the element is in the kernel
+                const uint32_t mag = words[k] & 0x7FFF7FFFu;
+                const float2 th = __fmul2_rn(ah2, b2[k]);                     // s_ij / 2 (exact halving of fl32(a_i b_j))
+                const uint32_t dc = floor16x2<DT>(th.x, th.y) + 0x80008000u - mag;
+                m_c |= (dc & 0x80008000u) >> k;
+                if constexpr (DUAL) m_p |= ((tpt2 + 0x80008000u - mag) & 0x80008000u) >> k;
+                uint32_t gone;
+                if constexpr (SAME) {
+                    gone = sign_halves(dc);                                   // 0xFFFF in the halves whose bit 15 is set
+                } else {
+                    const uint32_t bit = 0x00010001u << k;
+                    const float2 x = unpack16x2<DT>(words[k]);
+                    const float2 p = __fmul2_rn(x, rb2[k]);
+                    const float g0 = __fadd_rn(fabsf(p.x), -thr[2]), g1 = __fadd_rn(fabsf(p.y), -thr[2]);
                     near_g = fminf(near_g, fminf(fabsf(g0), fabsf(g1)));
                     gone = negative_halves(g0, g1);
                     m_g |= gone & bit;
                 }
-                if constexpr (DUAL) {
-                    const float e0 = __fadd_rn(fabsf(x.x), -thr[2]), e1 = __fadd_rn(fabsf(x.y), -thr[2]);
-                    near_p = fminf(near_p, fminf(fabsf(e0), fabsf(e1)));
-                    m_p |= negative_halves(e0, e1) & bit;
-                }
                 ow[k] = words[k] & ~gone;
             }
             unsigned int r_cq = __popc(m_c), r_pt = __popc(m_p), r_rm = SAME ? r_cq : __popc(m_g);
-            // (a NaN distance -- infinite threshold, band of zero -- compares false, exactly as the per-element test did)
-            bool undecided = !cols_trusted || near_c < thr[1];
-            if constexpr (!SAME) undecided |= near_g < thr[5];
-            if constexpr (DUAL) undecided |= near_p < thr[3];
+            // rows and columns whose scale factors are outside [2^-40, 2^40] (markers), and for a scaled bound the
+            // elements inside its band, go to the IEEE quotients
+            bool undecided = !cols_trusted || !(thr[0] == thr[0]);
+            if constexpr (DUAL) undecided |= tpt2 == 0xFFFFFFFFu;
+            if constexpr (!SAME) undecided |= near_g < thr[3];
             if (undecided) {
                 // Rare: some element sits within 2^-16 (relative) of a bound, or a scale factor is extreme.
                 // The whole vector is decided again from the IEEE quotients.
@@ -182,27 +223,34 @@ k9_zero_tests(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
         };
         // Lane l holds threshold number l / 4 (order of thr[] above) of row l % 4 of the group.  The scale is
         // fetched one group ahead (load_scale) and turned into the threshold when its group comes up.
-        constexpr int kKinds = !DUAL ? 2 : (SAME ? 4 : 6);
+        constexpr int kKinds = SAME ? (DUAL ? 2 : 1) : 4;
         const int kind = lane >> 2;
-        const bool per_token = kind == 2 || kind == 3;
-        const bool is_mid = (kind & 1) == 0;
-        float factor = zf.f[0];
-#pragma unroll
-        for (int k = 1; k < kKinds; ++k) factor = kind == k ? zf.f[k] : factor;
         auto load_scale = [&](int64_t g) {
             if (kind >= kKinds) return 0.0f;
             const int64_t row = min((g << 2) + (lane & 3), T - 1);
-            return per_token ? __ldg(t + row) : __ldg(a + row);
+            return kind == 1 ? __ldg(t + row) : __ldg(a + row);
         };
         auto threshold_of = [&](float raw) {
-            const float sc = (DUAL && per_token) ? __fmul_rn(raw, zf.inv_qmax) : raw;      // range check only
+            const float nan = __int_as_float(0x7FC00000);
+            if (kind == 0) {                                           // a_i / 2; a zero row has only zeros, which 0 admits
+                if (raw == 0.0f) return 0.0f;
+                return (raw >= kScaleLo && raw <= kScaleHi) ? __fmul_rn(0.5f, raw) : nan;
+            }
+            if (kind == 1) {                                           // per-token: largest 16-bit value <= fl32(t_i / qmax) / 2
+                if (raw == 0.0f) return 0.0f;
+                const float spt = __fdiv_rn(raw, qmaxf);
+                if (!(spt >= kScaleLo && spt <= kScaleHi)) return __uint_as_float(0xFFFFFFFFu);
+                const float h = __fmul_rn(0.5f, spt);
+                return __uint_as_float(floor16x2<DT>(h, h));
+            }
+            const bool is_mid = kind == 2;                             // (m, e) of the caller's bound, as before
             if (raw == 0.0f) return is_mid ? INFINITY : 0.0f;
-            if (sc >= kScaleLo && sc <= kScaleHi) return __fmul_rn(factor, raw);
+            if (raw >= kScaleLo && raw <= kScaleHi) return __fmul_rn(is_mid ? zf.m : zf.e, raw);
             return is_mid ? 0.0f : INFINITY;
         };
-        auto row_thresholds = [&](float tv, int u, float (&thr)[6]) {
+        auto row_thresholds = [&](float tv, int u, float (&thr)[4]) {
 #pragma unroll
-            for (int k = 0; k < 6; ++k) thr[k] = k < kKinds ? __shfl_sync(0xFFFFFFFFu, tv, 4 * k + u) : 0.0f;
+            for (int k = 0; k < 4; ++k) thr[k] = k < kKinds ? __shfl_sync(0xFFFFFFFFu, tv, 4 * k + u) : 0.0f;
         };
 
         if ((T & 3) != 0 && blockIdx.y == 0 && warp_active) {            // ragged last group
@@ -210,7 +258,7 @@ k9_zero_tests(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
             for (int u = 0; u < static_cast<int>(T & 3); ++u) {
                 const int64_t row = (nfull << 2) + u;
                 const uint4 slot = ld_stream(xp + row * ld8);
-                float thr[6];
+                float thr[4];
                 row_thresholds(tv, u, thr);
                 do_row(slot, thr, row, static_cast<int>(row * I8 + vv));
             }
@@ -235,7 +283,7 @@ k9_zero_tests(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8,
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const uint4 cur = stage[(st * 4 + u) * Wv + tid];
-                    float thr[6];
+                    float thr[4];
                     row_thresholds(tv, u, thr);
                     do_row(cur, thr, (g << 2) + u, vec + u * I8);
                 }
@@ -293,21 +341,15 @@ g9_zero_tests(const uint16_t* __restrict__ X, int64_t T, int64_t I, int64_t ld, 
 }
 
 // ============================================================================ host side
-static ZeroFactors factors_of(float h, float qmaxf) {
-    auto pair = [](float bound, float div, float* out) {
-        if (bound >= 9.5367431640625e-07f && bound <= 1048576.0f) {   // [2^-20, 2^20]
-            out[0] = bound / div;
-            out[1] = bound * 3.814697265625e-06f / div;               // 2^-18
-        } else {
-            out[0] = 0.0f;
-            out[1] = INFINITY;
-        }
-    };
+static ZeroFactors factors_of(float h) {
     ZeroFactors z{};
-    pair(0.5f, 1.0f, z.f);
-    pair(0.5f, qmaxf, z.f + 2);
-    pair(h, 1.0f, z.f + 4);
-    z.inv_qmax = 1.0f / qmaxf;
+    if (h >= 9.5367431640625e-07f && h <= 1048576.0f) {              // [2^-20, 2^20]
+        z.m = h;
+        z.e = h * 3.814697265625e-06f;                                // 2^-18
+    } else {
+        z.m = 0.0f;
+        z.e = INFINITY;
+    }
     return z;
 }
 
@@ -345,7 +387,7 @@ static bool launch_k9(const Plan& p, const ZeroArgs& z, cudaStream_t st) {
     if (y > 65535) y = 65535;
     if (y < 1) y = 1;
     launch_after(kern, dim3(p.nstrips, static_cast<unsigned>(y)), dim3(p.W), smem, st, static_cast<const uint4*>(z.X), z.T,
-                 p.I8, z.ld / 8, z.t, z.a, z.b, z.rb, z.qmaxf, z.half_bound, factors_of(z.half_bound, z.qmaxf),
+                 p.I8, z.ld / 8, z.t, z.a, z.b, z.rb, z.qmaxf, z.half_bound, factors_of(z.half_bound),
                  static_cast<uint4*>(z.out), z.counts);
     return true;
 }
