@@ -354,6 +354,25 @@ def test_rows_full_of_exact_ties(cq, bits, top):
             assert ties.mean() > 0.3
 
 
+@pytest.mark.parametrize("scale", [1e36, 1e-36, 3e-39, 2.0 ** -41, 2.0 ** 41])
+def test_weight_scales_outside_the_exact_quotient_range(cq, scale):
+    """Row and group scales beyond [2^-40, 2^40] (down to subnormal ones) leave the division-free quotient and take the
+    defining sequence; rows inside the range sit next to them in the same matrix."""
+    for bits in (8, 4):
+        W = wl.small_matrix(12, 1024, "bf16", 63, scale=scale, outlier_cols=2, outlier_scale=4.0, zero_frac=0.02)
+        W[3] = wl.small_matrix(1, 1024, "bf16", 64, scale=0.02)[0]            # an ordinary row among the extreme ones
+        W[7, :] = 0
+        Wd = to_dev(W, "bf16")
+        ref = orc.quantize_weight_per_channel(W, "bf16", bits)
+        r = cq.quantize_weight_per_channel(Wd, bits)
+        parity.check_weight(W, "bf16", bits, scale=r.scale.cpu().numpy(), codes=r.codes.cpu().numpy(), deq=bits_of(r.deq),
+                            zero_count=int(r.zero_count.item()), ref=ref)
+        refg = orc.quantize_weight_groupwise(W, "bf16", bits, 128)
+        g = cq.quantize_weight_groupwise(Wd, 128, bits)
+        parity.check_weight(W, "bf16", bits, scale=g.scale.cpu().numpy(), codes=g.codes.cpu().numpy(), deq=bits_of(g.deq),
+                            zero_count=int(g.zero_count.item()), ref=refg)
+
+
 def test_weight_groupwise_rejects_a_group_that_does_not_divide_the_row(cq):
     Wd = torch.zeros((4, 100), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(cq.CQError) as e:
