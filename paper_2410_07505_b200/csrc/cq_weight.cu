@@ -153,44 +153,64 @@ g4_weight_rows(const uint16_t* __restrict__ W, int64_t C, int64_t ld, int bits,
 }
 
 // ============================================================================ dequantize
-// One thread per 8 codes.  ODT: CQ_F16 / CQ_BF16 / CQ_F32.
+// Grid x = blocks of 256 vector columns (8 codes each), grid y = groups of kDeqRows rows (looped when there are more
+// groups than the grid may have).  A thread keeps the scale factors of its eight columns and handles the same
+// vector column in kDeqRows consecutive rows: all its code loads are issued before the first is used.
+// ODT: CQ_F16 / CQ_BF16 / CQ_F32.
+constexpr int kDeqRows = 4;
+
 template <int BITS, int ODT>
 __global__ void __launch_bounds__(kThreads)
 k5_dequantize(const void* __restrict__ codes, int64_t T, int I8, const float* __restrict__ a,
               const float* __restrict__ b, void* __restrict__ out) {
-    const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (idx >= T * I8) return;
-    const int64_t row = idx / I8;
-    const int v = static_cast<int>(idx % I8);
-    int q[8];
-    if constexpr (BITS == 8) {
-        uint2 w = __ldcs(reinterpret_cast<const uint2*>(codes) + idx);
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            q[e] = static_cast<int8_t>((w.x >> (8 * e)) & 0xFF);
-            q[4 + e] = static_cast<int8_t>((w.y >> (8 * e)) & 0xFF);
-        }
-    } else {
-        uint32_t w = __ldcs(reinterpret_cast<const uint32_t*>(codes) + idx);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) q[e] = (static_cast<int>(w << (28 - 4 * e))) >> 28;
-    }
-    const float ai = __ldg(a + row);
+    const int v = blockIdx.x * blockDim.x + threadIdx.x;
+    if (v >= I8) return;
     const float4 b0 = __ldg(reinterpret_cast<const float4*>(b) + 2 * v);
     const float4 b1 = __ldg(reinterpret_cast<const float4*>(b) + 2 * v + 1);
     const float bj[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-    float d[8];
+    const int64_t ngroups = (T + kDeqRows - 1) / kDeqRows;
+    for (int64_t g = blockIdx.y; g < ngroups; g += gridDim.y) {
+        const int64_t r0 = g * kDeqRows;
+        uint2 w8[kDeqRows];
+        uint32_t w4[kDeqRows];
+        float ai[kDeqRows];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) d[e] = __fmul_rn(static_cast<float>(q[e]), __fmul_rn(ai, bj[e]));
-    if constexpr (ODT == CQ_F32) {
-        float4* o = reinterpret_cast<float4*>(out) + idx * 2;
-        st_stream(o, make_float4(d[0], d[1], d[2], d[3]));
-        st_stream(o + 1, make_float4(d[4], d[5], d[6], d[7]));
-    } else {
-        uint4 o;
-        o.x = pack16x2<ODT>(d[0], d[1]); o.y = pack16x2<ODT>(d[2], d[3]);
-        o.z = pack16x2<ODT>(d[4], d[5]); o.w = pack16x2<ODT>(d[6], d[7]);
-        st_stream(reinterpret_cast<uint4*>(out) + idx, o);
+        for (int u = 0; u < kDeqRows; ++u) {
+            const int64_t row = r0 + u < T ? r0 + u : T - 1;          // rows past the end re-read the last one, store nothing
+            const int64_t idx = row * I8 + v;
+            if constexpr (BITS == 8) w8[u] = __ldcs(reinterpret_cast<const uint2*>(codes) + idx);
+            else w4[u] = __ldcs(reinterpret_cast<const uint32_t*>(codes) + idx);
+            ai[u] = __ldg(a + row);
+        }
+#pragma unroll
+        for (int u = 0; u < kDeqRows; ++u) {
+            if (r0 + u >= T) break;
+            const int64_t idx = (r0 + u) * I8 + v;
+            int q[8];
+            if constexpr (BITS == 8) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    q[e] = static_cast<int8_t>((w8[u].x >> (8 * e)) & 0xFF);
+                    q[4 + e] = static_cast<int8_t>((w8[u].y >> (8 * e)) & 0xFF);
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) q[e] = (static_cast<int>(w4[u] << (28 - 4 * e))) >> 28;
+            }
+            float d[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) d[e] = __fmul_rn(static_cast<float>(q[e]), __fmul_rn(ai[u], bj[e]));
+            if constexpr (ODT == CQ_F32) {
+                float4* o = reinterpret_cast<float4*>(out) + idx * 2;
+                st_stream(o, make_float4(d[0], d[1], d[2], d[3]));
+                st_stream(o + 1, make_float4(d[4], d[5], d[6], d[7]));
+            } else {
+                uint4 o;
+                o.x = pack16x2<ODT>(d[0], d[1]); o.y = pack16x2<ODT>(d[2], d[3]);
+                o.z = pack16x2<ODT>(d[4], d[5]); o.w = pack16x2<ODT>(d[6], d[7]);
+                st_stream(reinterpret_cast<uint4*>(out) + idx, o);
+            }
+        }
     }
 }
 
@@ -228,6 +248,7 @@ k6_count_zero_codes(const uint8_t* __restrict__ codes, int bits, int64_t head, i
     const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
     unsigned int zeros = 0;
     const uint4* vec = reinterpret_cast<const uint4*>(codes + head);
+#pragma unroll 4
     for (int64_t k = idx; k < body; k += stride) {
         uint4 w = __ldcs(vec + k);
         if (bits == 8) zeros += zero_bytes(w.x) + zero_bytes(w.y) + zero_bytes(w.z) + zero_bytes(w.w);
@@ -330,8 +351,9 @@ int cq_dequantize(const void* codes, int bits, int64_t T, int64_t I, const float
     const bool fast = (I % 8 == 0) && aligned(codes, bits == 8 ? 8 : 4) && aligned(col_scale, 16) && aligned(out, 16);
     if (fast) {
         const int I8 = static_cast<int>(I / 8);
-        const int64_t n = T * I8;
-        const unsigned blocks = static_cast<unsigned>((n + kThreads - 1) / kThreads);
+        const int64_t ngroups = (T + kDeqRows - 1) / kDeqRows;
+        const dim3 blocks(static_cast<unsigned>((I8 + kThreads - 1) / kThreads),
+                          static_cast<unsigned>(ngroups < 65535 ? ngroups : 65535));
 #define CQ_K5(B, O) k5_dequantize<B, O><<<blocks, kThreads, 0, st>>>(codes, T, I8, row_scale, col_scale, out)
         if (bits == 8) {
             if (out_dtype == CQ_F16) CQ_K5(8, CQ_F16); else if (out_dtype == CQ_BF16) CQ_K5(8, CQ_BF16); else CQ_K5(8, CQ_F32);

@@ -101,6 +101,10 @@ def time_extra_ops(Xd: torch.Tensor, alpha: float, flush, iters: int) -> dict:
     us_cnt = _time(lambda: cq.kernel_count_x(Xd, alpha, 8, t, c, ws), flush.read, iters)
     us_abs = _time(lambda: cq.absmax_rows_cols(Xd), flush.read, iters)
     us_abs_ws = _time(lambda: cq.absmax_rows_cols(Xd, workspace=ws, out=(t, c)), flush.read, iters)
+    deq = torch.empty((T, I), dtype=Xd.dtype, device=Xd.device)
+    cnt = torch.zeros((), dtype=torch.int64, device=Xd.device)
+    us_deq = _time(lambda: cq.dequantize(r.codes, 8, T, I, r.row_scale, r.col_scale, Xd.dtype, out=deq), flush.read, iters)
+    us_kc = _time(lambda: cq.kernel_count(r.codes, 8, T, I, count=cnt), flush.read, iters)
     _, counts = cq.remove_kernel(Xd, alpha, 8, 1.0, ws)
     ind = cq.case_indicators(r).cpu().tolist()
     cnt = counts.cpu().tolist()
@@ -108,6 +112,8 @@ def time_extra_ops(Xd: torch.Tensor, alpha: float, flush, iters: int) -> dict:
             "case_indicators_us": round(us_ind, 1), "kernel_count_x_us": round(us_cnt, 1),
             "absmax_rows_cols_us": round(us_abs, 1), "absmax_gbs": round(2 * n / us_abs / 1e3, 1),
             "absmax_with_workspace_us": round(us_abs_ws, 1),
+            "dequantize_us": round(us_deq, 1), "dequantize_gbs": round(3 * n / us_deq / 1e3, 1),
+            "kernel_count_us": round(us_kc, 1), "kernel_count_gbs": round(n / us_kc / 1e3, 1),
             "kernel_proportion_per_token": cnt[1] / n, "kernel_proportion_crossquant": cnt[2] / n,
             "share_c_ge_t": ind[0] / n, "share_bound_smaller": ind[1] / n}
 
