@@ -254,7 +254,7 @@ int cq_case_indicators(const float* t, const float* c, const float* row_scale, c
  *   "no_pdl"      1: no programmatic dependent launch (quantize pass and diagnostics passes)
  *   "no_stage"    1: the quantize pass loads rows straight into registers instead of staging them in shared memory
  *                    with bulk copies; the weight quantizer uses plain loads for long rows too
- *   "no_small"    1: decode-sized matrices (up to 8192 columns and 16-32 rows) take the three launches too
+ *   "no_small"    1: decode-sized matrices (up to 8192 columns and 16-256 rows) take the three launches too
  *                    instead of the single thread-block-cluster launch
  * value <= 0 restores the built-in choice.  Returns CQ_OK or CQ_ERR_SHAPE (unknown key). */
 int cq_set_tuning(const char* key, int value);

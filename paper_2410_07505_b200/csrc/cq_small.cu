@@ -17,7 +17,8 @@ namespace cg = cooperative_groups;
 
 namespace cq {
 
-constexpr int kSmallRows = 4;
+constexpr int kSmallRows = 16;        // most rows of a tile one CTA may hold
+constexpr int kSmallTileVecs = 1024;  // most 8-element vectors of a tile (4 rows of a full strip, 8-16 rows of a narrow one)
 __device__ unsigned int g_small_stage_fault = 0;      // set if the bounded wait on the tile copy ever gave up
 constexpr int kSmallStrips = 4;       // more column strips would leave each thread more than two pows
 
@@ -146,10 +147,13 @@ k_small(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8, int Tc, dou
     }
     const bool cols_trusted = ((rb2[0].x + rb2[0].y) + (rb2[1].x + rb2[1].y)) +
                               ((rb2[2].x + rb2[2].y) + (rb2[3].x + rb2[3].y)) < INFINITY;
-    cluster.sync();                                               // nobody reads this CTA's shared memory any more (and s_a / s_ra are in place)
+    // This CTA has read all it needs from the others; it may not exit before they have read what they need from it.
+    // Arrive now, wait at the end: the quantize phase runs meanwhile (s_a / s_ra were in place at the barrier above).
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
 
     // ---- quantize the tile from shared memory
     unsigned int zeros = 0;
+#pragma unroll 2
     for (int r = 0; r < rows; ++r) {
         const uint4 w = active ? s_x[r * Wv + tid] : make_uint4(0, 0, 0, 0);
         const float au = s_a[r], rau = s_ra[r];
@@ -184,6 +188,7 @@ k_small(const uint4* __restrict__ X, int64_t T, int I8, int64_t ld8, int Tc, dou
         }
     }
     if (zero_count != nullptr) cta_count_add(zeros, zero_count);
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
 template <int DT, int BITS>
@@ -230,10 +235,16 @@ int small_stage_fault(unsigned int* fault_host) {
 
 bool launch_small(const SmallArgs& s, cudaStream_t st) {
     if (s.nstrips < 1 || s.nstrips > kSmallStrips || s.T < 1) return false;
-    // row chunks: as many as the cluster has room for (a chunk may be empty: its CTA still takes its share of the pows)
-    const int RY = (s.nstrips <= 2 ? 8 : 16) / s.nstrips;
-    const int64_t Tc64 = (s.T + RY - 1) / RY;
-    if (Tc64 > kSmallRows) return false;
+    // row chunks: as many as the cluster has room for (a chunk may be empty: its CTA still takes its share of the pows);
+    // one or two strips go from the portable 8-CTA cluster to 16 CTAs when that is what makes the tile small enough
+    auto fits = [&](int64_t tc) { return tc <= kSmallRows && tc * s.W <= kSmallTileVecs; };
+    int RY = (s.nstrips <= 2 ? 8 : 16) / s.nstrips;
+    int64_t Tc64 = (s.T + RY - 1) / RY;
+    if (!fits(Tc64) && s.nstrips <= 2) {
+        RY = 16 / s.nstrips;
+        Tc64 = (s.T + RY - 1) / RY;
+    }
+    if (!fits(Tc64)) return false;
     const int Tc = static_cast<int>(Tc64);
     if (s.dtype == CQ_F16)
         return s.bits == 8 ? launch_small_typed<CQ_F16, 8>(s, RY, Tc, st) : launch_small_typed<CQ_F16, 4>(s, RY, Tc, st);

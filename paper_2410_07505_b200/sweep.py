@@ -151,7 +151,7 @@ def time_decode_shapes(flush, iters: int) -> None:
     """Decode-sized matrices: CUDA-event time of one call after an L2 flush, wall time per call of 200 calls issued
     back to back (host included), for the single-launch path and the three launches, and per replay of a graph."""
     import time
-    for T, I in ((1, 4096), (16, 4096), (16, 8192), (32, 2048), (64, 8192)):
+    for T, I in ((1, 4096), (16, 4096), (16, 8192), (32, 2048), (128, 768), (64, 2048), (32, 4096), (64, 8192)):
         Xd = _dev(wl.small_matrix(T, I, "bf16", 3, outlier_cols=4), "bf16")
         buf = cq.ActBuffers(T, I, Xd.dtype, 8)
         row = {"shape": [T, I], "dtype": "bf16", "bits": 8}

@@ -153,14 +153,19 @@ def test_tiling_knobs_do_not_change_results(cq):
 
 
 SMALL_SHAPES = [(1, 8), (1, 4096), (3, 16), (16, 4096), (16, 8192), (32, 2048), (31, 776), (9, 5000), (5, 8200), (16, 6152),
-                (33, 2048), (17, 8192)]
+                (33, 2048), (17, 8192),
+                # narrow strips hold more rows per cluster CTA (up to 16, up to 1024 vectors per tile); one or two strips
+                # may take a 16-CTA cluster: shapes at and just past those limits
+                (128, 768), (129, 768), (256, 256), (250, 200), (257, 256), (64, 2048), (65, 2048), (32, 4096), (33, 4096),
+                (160, 512), (161, 520)]
 
 
 @pytest.mark.parametrize("shape", SMALL_SHAPES)
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
 def test_small_matrices_one_launch_and_three_launches(cq, shape, dtype):
-    """Decode-sized matrices take a single thread-block-cluster launch (up to 4 rows per cluster CTA, up to four
-    column strips); the shapes around its limits and the same shapes forced through the three launches."""
+    """Decode-sized matrices take a single thread-block-cluster launch (4 rows of a full strip to 16 rows of a narrow one
+    per cluster CTA, up to four column strips); the shapes around its limits and the same shapes forced through the
+    three launches."""
     T, I = shape
     X = wl.small_matrix(T, I, dtype, 700 + T + I, outlier_cols=3, outlier_scale=30.0, zero_frac=0.03)
     X[0, : min(I, 24)] = 0
