@@ -248,12 +248,18 @@ k6_count_zero_codes(const uint8_t* __restrict__ codes, int bits, int64_t head, i
     const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
     unsigned int zeros = 0;
     const uint4* vec = reinterpret_cast<const uint4*>(codes + head);
-#pragma unroll 4
-    for (int64_t k = idx; k < body; k += stride) {
-        uint4 w = __ldcs(vec + k);
-        if (bits == 8) zeros += zero_bytes(w.x) + zero_bytes(w.y) + zero_bytes(w.z) + zero_bytes(w.w);
-        else zeros += zero_nibbles(w.x) + zero_nibbles(w.y) + zero_nibbles(w.z) + zero_nibbles(w.w);
+    auto count16 = [bits](const uint4& w) -> unsigned int {
+        if (bits == 8) return zero_bytes(w.x) + zero_bytes(w.y) + zero_bytes(w.z) + zero_bytes(w.w);
+        return zero_nibbles(w.x) + zero_nibbles(w.y) + zero_nibbles(w.z) + zero_nibbles(w.w);
+    };
+    // four independent 16-byte loads per thread and round, all issued before the first is used
+    int64_t k = idx;
+    for (; k + 3 * stride < body; k += 4 * stride) {
+        const uint4 w0 = __ldcs(vec + k), w1 = __ldcs(vec + k + stride), w2 = __ldcs(vec + k + 2 * stride),
+                    w3 = __ldcs(vec + k + 3 * stride);
+        zeros += count16(w0) + count16(w1) + count16(w2) + count16(w3);
     }
+    for (; k < body; k += stride) zeros += count16(__ldcs(vec + k));
     auto byte_zeros = [bits](uint8_t v) -> unsigned int {
         if (bits == 8) return v == 0;
         return ((v & 0xF) == 0) + ((v >> 4) == 0);
