@@ -259,7 +259,9 @@ def test_absmax_entry_points(cq, shape, dtype):
     assert np.array_equal(cq.absmax_cols(Xd).cpu().numpy(), c_ref)
 
 
-@pytest.mark.parametrize("shape", [(65, 512), (33, 50), (9, 1030)])
+# (262147, 8): more groups of four rows than a grid may have in y (the kernel loops); (7, 4104): three blocks of vector
+# columns, the last one ragged, and a ragged last row group
+@pytest.mark.parametrize("shape", [(65, 512), (33, 50), (9, 1030), (262147, 8), (7, 4104)])
 @pytest.mark.parametrize("bits", [8, 4])
 def test_dequantize_and_kernel_count_from_stored_codes(cq, shape, bits):
     T, I = shape
