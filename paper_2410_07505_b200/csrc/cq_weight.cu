@@ -153,23 +153,29 @@ g4_weight_rows(const uint16_t* __restrict__ W, int64_t C, int64_t ld, int bits,
 }
 
 // ============================================================================ dequantize
-// Grid x = blocks of 256 vector columns (8 codes each), grid y = groups of kDeqRows rows (looped when there are more
-// groups than the grid may have).  A thread keeps the scale factors of its eight columns and handles the same
+// Block = (W vector columns of 8 codes) x (256 / W row groups), W = 256 or, for narrower matrices, the power of two that
+// covers the row; grid x = blocks of W vector columns, grid y = blocks of row groups of kDeqRows rows (looped when there
+// are more than the grid may have).  A thread keeps the scale factors of its eight columns and handles the same
 // vector column in kDeqRows consecutive rows: all its code loads are issued before the first is used.
 // ODT: CQ_F16 / CQ_BF16 / CQ_F32.
 constexpr int kDeqRows = 4;
 
-template <int BITS, int ODT>
+// NARROW: rows shorter than 256 vectors, several row groups per block (the group then differs from thread to thread;
+// with one group per block its row scales and addresses stay uniform across the block, which halves the registers).
+template <int BITS, int ODT, bool NARROW>
 __global__ void __launch_bounds__(kThreads)
 k5_dequantize(const void* __restrict__ codes, int64_t T, int I8, const float* __restrict__ a,
               const float* __restrict__ b, void* __restrict__ out) {
     const int v = blockIdx.x * blockDim.x + threadIdx.x;
     if (v >= I8) return;
+    const int g0 = NARROW ? blockIdx.y * blockDim.y + threadIdx.y : blockIdx.y;          // at most 65535 * 256
+    const int gstep = NARROW ? gridDim.y * blockDim.y : gridDim.y;
     const float4 b0 = __ldg(reinterpret_cast<const float4*>(b) + 2 * v);
     const float4 b1 = __ldg(reinterpret_cast<const float4*>(b) + 2 * v + 1);
     const float bj[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
     const int64_t ngroups = (T + kDeqRows - 1) / kDeqRows;
-    for (int64_t g = blockIdx.y; g < ngroups; g += gridDim.y) {
+#pragma unroll 1
+    for (int64_t g = g0; g < ngroups; g += gstep) {
         const int64_t r0 = g * kDeqRows;
         uint2 w8[kDeqRows];
         uint32_t w4[kDeqRows];
@@ -358,9 +364,16 @@ int cq_dequantize(const void* codes, int bits, int64_t T, int64_t I, const float
     if (fast) {
         const int I8 = static_cast<int>(I / 8);
         const int64_t ngroups = (T + kDeqRows - 1) / kDeqRows;
-        const dim3 blocks(static_cast<unsigned>((I8 + kThreads - 1) / kThreads),
-                          static_cast<unsigned>(ngroups < 65535 ? ngroups : 65535));
-#define CQ_K5(B, O) k5_dequantize<B, O><<<blocks, kThreads, 0, st>>>(codes, T, I8, row_scale, col_scale, out)
+        int W = kThreads;
+        while (W / 2 >= I8 && W > 1) W /= 2;
+        const dim3 threads(static_cast<unsigned>(W), static_cast<unsigned>(kThreads / W));
+        const int64_t gblocks = (ngroups + threads.y - 1) / threads.y;
+        const dim3 blocks(static_cast<unsigned>((I8 + W - 1) / W), static_cast<unsigned>(gblocks < 65535 ? gblocks : 65535));
+#define CQ_K5(B, O)                                                                                        \
+    do {                                                                                                   \
+        if (W < kThreads) k5_dequantize<B, O, true><<<blocks, threads, 0, st>>>(codes, T, I8, row_scale, col_scale, out);  \
+        else k5_dequantize<B, O, false><<<blocks, threads, 0, st>>>(codes, T, I8, row_scale, col_scale, out);             \
+    } while (0)
         if (bits == 8) {
             if (out_dtype == CQ_F16) CQ_K5(8, CQ_F16); else if (out_dtype == CQ_BF16) CQ_K5(8, CQ_BF16); else CQ_K5(8, CQ_F32);
         } else {

@@ -284,6 +284,22 @@ def test_dequantize_and_kernel_count_from_stored_codes(cq, shape, bits):
         assert int(cq.kernel_count(pad[3:], bits, T, I).item()) == ref.zero_count
 
 
+def test_dequantize_more_row_groups_than_grid_rows(cq):
+    """262,150 rows of 1032 codes: 65,538 groups of four rows, more than a grid may have in y, so the kernel loops.
+    Row blocks of the result (the first, one across the grid limit, the ragged last) must equal what separate calls
+    on those rows alone give (small calls of this kind are compared with the oracle above)."""
+    T, I = 262150, 1032
+    g = torch.Generator(device="cuda").manual_seed(5)
+    codes = torch.randint(-127, 128, (T, I), dtype=torch.int8, device="cuda", generator=g)
+    a = torch.rand(T, device="cuda", generator=g) + 0.01
+    b = torch.rand(I, device="cuda", generator=g) + 0.01
+    out = cq.dequantize(codes, 8, T, I, a, b, torch.bfloat16)
+    for lo, hi in ((0, 9), (4 * 65535 - 3, 4 * 65535 + 5), (T - 6, T)):
+        part = cq.dequantize(codes[lo:hi].contiguous(), 8, hi - lo, I, a[lo:hi].contiguous(), b, torch.bfloat16)
+        assert torch.equal(out[lo:hi].view(torch.int16), part.view(torch.int16))
+    assert int(cq.kernel_count(codes, 8, T, I).item()) == int((codes == 0).sum().item())
+
+
 @pytest.mark.parametrize("bits", [8, 4])
 def test_kernel_count_straight_from_x(cq, bits):
     X = wl.small_matrix(200, 1032, "f16", 41, outlier_cols=4, outlier_scale=40.0, zero_frac=0.01)
