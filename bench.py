@@ -324,13 +324,17 @@ def main() -> None:
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
-    with clk.ClockSampler(local, str(torch.cuda.get_device_properties(local).uuid), period_s=0.002) as clocks:
+    # the SM clock and the throttle reasons are sampled (NVML, every 0.5 ms) while the timed steps run and, further
+    # down, while the hooked launches of the roofline object run: both are the load the reported numbers come from
+    clocks = clk.ClockSampler(local, str(torch.cuda.get_device_properties(local).uuid), period_s=0.0005)
+    with clocks:
         for k in range(K):
             flush_l2("read")                      # untimed: evicts X and the outputs from L2
             ev[k][0].record()
             step()
             ev[k][1].record()
         torch.cuda.synchronize()
+    step_samples, step_reasons = list(clocks.samples), set(clocks.reasons)
     if world > 1:
         dist.barrier()
     step_ms = [e[0].elapsed_time(e[1]) for e in ev]
@@ -345,12 +349,15 @@ def main() -> None:
         a_.record()
         b_.record()
     torch.cuda.synchronize()
-    for a_, b_ in hook:
-        flush_l2("read")
-        cq.set_timing_events(a_, b_)
-        step()
-    torch.cuda.synchronize()
+    with clocks:
+        for a_, b_ in hook:
+            flush_l2("read")
+            cq.set_timing_events(a_, b_)
+            step()
+        torch.cuda.synchronize()
     cq.set_timing_events(None, None)
+    clocks.samples = step_samples + clocks.samples
+    clocks.reasons |= step_reasons
     quant_ms = [a_.elapsed_time(b_) for a_, b_ in hook]
 
     # ---- end to end: host buffers in, host buffers out, through cq_quantize_act_host.
